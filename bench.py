@@ -1,0 +1,443 @@
+#!/usr/bin/env python
+"""Benchmark of the k-means LUT linear layer (libkmq) on B200.
+
+One "step" is one pass of the hot path over a pool of distinct weight sets:
+for every bit width of the workload, `kmq_linear` is called once per pool
+entry (different packed weights, codebooks, activations and outputs per call,
+pool larger than L2 so no call finds its weights cached -- the protocol of the
+paper's micro-benchmarks, Appendix "Benchmarking").  The calls of a step are
+captured in CUDA graphs and replayed; time is taken with CUDA events on the
+launching stream.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config2]
+    python bench.py --impl reference ...        # the CPU oracle on the host cores
+
+Prints ONE JSON line (rank 0).  `value` is algorithmic bytes per second:
+packed indices + codebooks + activations + outputs of every call, summed over
+all ranks, divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+# workload -> list of (layer name, N, K, distribution, bits, M)
+WORKLOADS = {
+    "config2": [("square4096", 4096, 4096, "normal", b, 1) for b in (1, 2, 4)],
+    "config3_m1": [(n, N, K, "student_t", 2, 1) for n, N, K in
+                   (("qkv", 9216, 3072), ("o", 3072, 3072), ("gate_up", 16384, 3072), ("down", 3072, 8192))],
+    "config3_m8": [(n, N, K, "student_t", 2, 8) for n, N, K in
+                   (("qkv", 9216, 3072), ("o", 3072, 3072), ("gate_up", 16384, 3072), ("down", 3072, 8192))],
+    "config4": [("square8192", 8192, 8192, "normal", 2, m) for m in (1, 2, 4, 8, 16, 32, 64)],
+    "config5": [("down_large", 8192, 28672, "laplace", b, m) for b in (1, 4) for m in (1, 16)],
+    "tiny": [("tiny", 256, 256, "normal", b, 1) for b in (1, 2, 4)],
+}
+WORKLOAD_TEXT = {
+    "config2": "single square layer N=K=4096, batch 1, b in {1,2,4}, per-row 2^b-centroid bf16 codebooks "
+               "(1-D Lloyd, 20 iterations) on N(0, 0.02) weights, bf16 N(0,1) activations",
+    "config3_m1": "3.9B-style decoder linear set (QKV 3072->9216, O 3072->3072, gate+up 3072->16384, "
+                  "down 8192->3072), b=2, batch 1, Student-t(5) weights",
+    "config3_m8": "3.9B-style decoder linear set, b=2, batch 8, Student-t(5) weights",
+    "config4": "batch sweep on N=K=8192, b=2, batch in {1,2,4,8,16,32,64}",
+    "config5": "large down projection N=8192 K=28672, b in {1,4}, batch in {1,16}, Laplace weights",
+    "tiny": "256x256 correctness layer",
+}
+CONFIG_ID = {"config2": 2, "config3_m1": 3, "config3_m8": 3, "config4": 4, "config5": 5, "tiny": 1}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel,
+# from the ncu capture summarised under profiles/ (None = not captured yet).
+NCU_TRAFFIC_BYTES = {}
+
+
+def algorithmic_bytes(N, K, bits, M):
+    return N * K * bits // 8 + N * (1 << bits) * 2 + M * K * 2 + M * N * 2
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------
+# clocks sampler (read-only NVML queries)
+# --------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index, period=0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons = [], set()
+        self.active = False
+        self.stop_flag = False
+        self.max_mhz = None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self.stop_flag:
+            try:
+                mhz = self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)
+                mask = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+            except Exception:
+                try:
+                    mask = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                except Exception:
+                    mask = 0
+                    mhz = None
+            if self.active and mhz is not None:
+                self.samples.append(mhz)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            time.sleep(self.period)
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------
+# the library arm
+# --------------------------------------------------------------------------
+class Case:
+    """One (layer, bits, M) of the workload with its pool of device buffers."""
+
+    def __init__(self, name, N, K, dist, bits, M, config_id, torch, kmq, synth, pool_bytes):
+        self.name, self.N, self.K, self.bits, self.M = name, N, K, bits, M
+        self.bytes = algorithmic_bytes(N, K, bits, M)
+        self.pool = max(4, -(-pool_bytes // self.bytes))
+        layer = synth.make_layer(N, K, bits, M, dist, config_id=config_id)
+        self.layer = layer
+        dev = torch.device("cuda")
+        idx = torch.from_numpy(layer["idx"]).to(dev)
+        words = kmq.kmq_packed_bytes(N, K, bits) // 4
+        self.packed = torch.empty((self.pool, words), dtype=torch.int32, device=dev)
+        kmq.kmq_pack(idx, N, K, bits, self.packed[0])              # a1: offline packing, on the GPU
+        self.packed[1:] = self.packed[0]
+        del idx
+        cb = torch.from_numpy(layer["codebooks"].view(np.int16)).to(dev)
+        self.cb = cb.unsqueeze(0).repeat(self.pool, 1, 1).contiguous()
+        rng = synth.rng_for(config_id, 100 + bits * 1000 + M)
+        xs = np.stack([layer["x"]] + [synth.draw_activations(M, K, rng) for _ in range(self.pool - 1)])
+        self.x_host = torch.from_numpy(xs.view(np.int16)).pin_memory()
+        self.x = self.x_host.to(dev)
+        self.y = torch.zeros((self.pool, M, N), dtype=torch.int16, device=dev)
+        self.y_host = torch.zeros((self.pool, M, N), dtype=torch.int16).pin_memory()
+        self.ws_bytes = kmq.kmq_workspace_bytes(N, K, bits, M)
+        self.ws = torch.empty(max(self.ws_bytes, 16), dtype=torch.uint8, device=dev)
+        self.launches = kmq.kmq_linear_num_launches(N, K, bits, M)
+        self.variant = kmq.kmq_linear_variant(N, K, bits, M)
+        self.kmq = kmq
+
+    def call(self, i):
+        self.kmq.kmq_linear(self.packed[i], self.cb[i], self.x[i], self.y[i], self.N, self.K, self.bits, self.M,
+                            self.ws, self.ws_bytes)
+
+    def call_host(self, i):
+        self.kmq.kmq_linear_host(self.packed[i], self.cb[i], self.x_host[i].data_ptr(), self.y_host[i].data_ptr(),
+                                 self.N, self.K, self.bits, self.M, self.x[i], self.y[i], self.ws, self.ws_bytes)
+
+
+def run_library(args):
+    import torch
+    from paper_2602_15563_b200 import build as kb
+    from paper_2602_15563_b200 import kmq, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libkmq has no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        kb.build()
+    if dist is not None:
+        dist.barrier()
+    kmq.lib()
+
+    peak_gbs, peak_kind = measured_peak()
+    cfg_id = CONFIG_ID[args.workload]
+    pool_bytes = 2 * L2_BYTES
+    cases = [Case(n, N, K, d, b, M, cfg_id, torch, kmq, synth, pool_bytes)
+             for (n, N, K, d, b, M) in WORKLOADS[args.workload]]
+
+    stream = torch.cuda.Stream()
+    graphs = []
+    with torch.cuda.stream(stream):
+        for c in cases:                       # warm every kernel outside capture first
+            c.call(0)
+        stream.synchronize()
+        for c in cases:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(c.pool):
+                    c.call(i)
+            graphs.append(g)
+
+    def one_step(events=None):
+        for j, g in enumerate(graphs):
+            if events is not None:
+                events[j][0].record(stream)
+            g.replay()
+            if events is not None:
+                events[j][1].record(stream)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            one_step()
+        barrier()
+        # ---- timed region: exactly K steps ----
+        ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in cases]
+              for _ in range(args.steps)]
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler.active = True
+        t0.record(stream)
+        for s in range(args.steps):
+            one_step(ev[s])
+        t1.record(stream)
+        barrier()
+        sampler.active = False
+    elapsed_ms = t0.elapsed_time(t1)
+    per_case_ms = [sum(ev[s][j][0].elapsed_time(ev[s][j][1]) for s in range(args.steps)) / args.steps
+                   for j in range(len(cases))]
+
+    step_bytes = sum(c.bytes * c.pool for c in cases)
+    step_calls = sum(c.pool for c in cases)
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    value = world * step_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9
+
+    # ---- end to end through the host-buffer entry point (H2D of x, D2H of y inside) ----
+    e2e_steps = max(1, min(args.steps, 5))
+    with torch.cuda.stream(stream):
+        for c in cases:
+            c.call_host(0)
+        barrier()
+        w0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            for c in cases:
+                for i in range(c.pool):
+                    c.call_host(i)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - w0
+    if dist is not None:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = world * step_bytes * e2e_steps / e2e_s / 1e9
+    h2d = sum(c.M * c.K * 2 * c.pool for c in cases)
+    d2h = sum(c.M * c.N * 2 * c.pool for c in cases)
+
+    sampler.stop_flag = True
+    sampler.join(timeout=1.0)
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- parity spot check of what was just timed (rank 0) ----
+    from oracle import kmq_oracle as orc
+    worst = 0.0
+    checked = 0
+    for c in cases:
+        ref_packed = orc.pack_canonical(c.layer["idx"], c.bits)
+        for i in sorted({0, c.pool - 1}):
+            x_i = c.x_host[i].numpy().view(np.uint16)
+            y_ref, s = orc.linear_f64(ref_packed, c.layer["codebooks"], x_i, c.K, c.bits)
+            y = c.y[i].cpu().numpy().view(np.uint16)
+            yh = c.y_host[i].numpy().view(np.uint16)
+            worst = max(worst, orc.check_linear(y, y_ref, s), orc.check_linear(yh, y_ref, s))
+            checked += 1
+
+    # ---- per-case figures and the roofline of the dominant kernel ----
+    per_case = []
+    for c, ms in zip(cases, per_case_ms):
+        us = ms * 1e3 / c.pool
+        gbs = c.bytes / (us * 1e-6) / 1e9
+        per_case.append({"layer": c.name, "N": c.N, "K": c.K, "bits": c.bits, "M": c.M, "pool": c.pool,
+                         "variant": c.variant, "us_per_call": round(us, 3), "gbs": round(gbs, 1),
+                         "frac_of_measured_hbm": round(gbs / peak_gbs, 4), "frac_of_8tbs": round(gbs / 8000.0, 4),
+                         "bytes_per_call": c.bytes})
+    dom = max(range(len(cases)), key=lambda j: per_case_ms[j])
+    dc = cases[dom]
+    achieved = per_case[dom]["gbs"] / dc.launches if dc.launches > 1 else per_case[dom]["gbs"]
+    roofline = {"bound": "hbm", "kernel": f"kmq_linear[{dc.variant}] b={dc.bits} M={dc.M} {dc.N}x{dc.K}",
+                "achieved": round(achieved, 1), "peak": peak_gbs, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": round(achieved / peak_gbs, 4),
+                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dc.bits, dc.M)),
+                "algorithmic_bytes_per_launch": dc.bytes}
+
+    cpu = cpu_baseline(args.workload, budget_s=args.cpu_seconds)
+
+    line = {
+        "metric": "kmq_linear effective HBM bandwidth (algorithmic bytes / time), batch-1 k-means LUT GEMV",
+        "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": round(elapsed_ms / args.steps, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {WORKLOAD_TEXT[args.workload]}",
+                   "calls_per_step": step_calls, "bytes_per_step": step_bytes,
+                   "l2": "inputs larger than L2: every call of a step uses its own weight set, pool >= 2 x 126 MB",
+                   "launch": "CUDA graph per case, replayed once per step", "multi_gpu": "replicas only"},
+        "frac_of_measured_hbm": round(value / world / peak_gbs, 4),
+        "us_per_call_mean": round(elapsed_ms * 1e3 / args.steps / step_calls, 3),
+        "per_case": per_case,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "e2e": {"value": round(e2e_value, 2), "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "api": "kmq_linear_host (x from pinned host memory, y back to host, per call)"},
+        "gpu_launches": args.steps * sum(c.pool * c.launches for c in cases),
+        "clocks": sampler.summary(),
+        "parity": {"calls_checked": checked, "max_err_over_tol": round(worst, 4), "ok": bool(worst <= 1.0)},
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------
+# the CPU oracle, timed (reported baseline and the reference arm)
+# --------------------------------------------------------------------------
+def _cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def _oracle_cases(workload):
+    from oracle import kmq_oracle as orc
+    from paper_2602_15563_b200 import synth
+    out = []
+    for (name, N, K, d, b, M) in WORKLOADS[workload]:
+        layer = synth.make_layer(N, K, b, M, d, config_id=CONFIG_ID[workload])
+        out.append((N, K, b, M, orc.pack_canonical(layer["idx"], b), layer["codebooks"], layer["x"]))
+    return out
+
+
+def cpu_baseline(workload, budget_s=12.0, cases=None):
+    """Time the oracle's inference part (unpack, table lookup, float64 matmul)
+    on the host cores, on a bounded sample of the workload."""
+    from oracle import kmq_oracle as orc
+    cases = cases or _oracle_cases(workload)
+    for (N, K, b, M, packed, cb, x) in cases[:1]:
+        orc.linear_f64(packed, cb, x, K, b)                       # warm-up
+    total_bytes, n_calls = 0, 0
+    t0 = time.perf_counter()
+    while True:
+        for (N, K, b, M, packed, cb, x) in cases:
+            orc.linear_f64(packed, cb, x, K, b)
+            total_bytes += algorithmic_bytes(N, K, b, M)
+            n_calls += 1
+        if time.perf_counter() - t0 >= budget_s or n_calls >= 1000:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": round(total_bytes / dt / 1e9, 4), "unit": "GB/s", "cores": _cpu_threads(),
+            "host_cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+            "sample": f"{n_calls} oracle calls ({n_calls // len(cases)} pass(es) over the {len(cases)} cases of "
+                      f"{workload}, one weight set each), {dt:.1f} s", "us_per_call": round(dt / n_calls * 1e6, 1)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from oracle import kmq_oracle as orc
+    cases = _oracle_cases(args.workload)
+    step_bytes = sum(algorithmic_bytes(N, K, b, M) for (N, K, b, M, *_r) in cases)
+
+    def step():
+        for (N, K, b, M, packed, cb, x) in cases:
+            orc.linear_f64(packed, cb, x, K, b)
+
+    steps = max(1, min(args.steps, 40))
+    for _ in range(max(1, min(args.warmup, 3))):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = step_bytes * steps / dt / 1e9
+    cores = _cpu_threads()
+    sample = f"one oracle call per case of {args.workload} per step ({len(cases)} calls), {steps} steps"
+    line = {
+        "impl": "reference",
+        "metric": "kmq_linear effective HBM bandwidth (algorithmic bytes / time), batch-1 k-means LUT GEMV",
+        "value": round(value, 4), "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": max(1, min(args.warmup, 3)),
+        "ms_per_step": round(dt / steps * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {WORKLOAD_TEXT[args.workload]}", "calls_per_step": len(cases),
+                   "bytes_per_step": step_bytes},
+        "cpu_baseline": {"value": round(value, 4), "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="kmq", choices=["kmq", "reference"])
+    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS))
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_library(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,135 @@
+/*
+ * libkmq -- k-means-quantised linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer is y = x * W^T with W^[n,k] = C_n[idx[n,k]]: every weight is a
+ * b-bit index (b = 1, 2 or 4) into the 2^b-entry bf16 codebook of its output
+ * row n.  This is the fused dequantise-multiply Y^T = dequantize(W~) X^T of
+ * the paper's Appendix "Benchmarking" ("Kernel implementations": gather the
+ * decoded values from a lookup table, then x @ W.T), with the lookup table
+ * held per output row and no block scales; the indices come from the
+ * nearest-centroid quantiser f_c(x) = argmin_i |x - c_i| (Section 2.1,
+ * "Rounding to nearest centroids").
+ *
+ * Conventions shared by every entry point
+ *   - Pointers marked DEVICE are CUDA device pointers valid on the current
+ *     device; HOST pointers are ordinary (ideally pinned) host memory.  The
+ *     caller owns every buffer.  The library allocates no memory and keeps no
+ *     state besides a per-device cache of device properties.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Work is enqueued on it and the call returns without synchronising,
+ *     unless stated otherwise.
+ *   - Arguments are validated on the host before anything is launched.  A
+ *     failed check returns a status and launches nothing.  Nothing aborts,
+ *     throws, or asserts on the device.
+ *   - bf16 values are passed as uint16_t bit patterns.
+ *   - Shapes: N output rows, K input features, M batch rows.  N, M >= 1;
+ *     K >= 32/bits and K % (32/bits) == 0.  Buffers must not overlap.
+ *   - Canonical packed layout (KMQ_LAYOUT_CANONICAL): row-major
+ *     uint32 [N, K*bits/32]; bits [i*bits, (i+1)*bits) of word j of row n hold
+ *     idx[n, j*(32/bits) + i] (fields LSB first, packed along K).
+ *   - All device pointers must be 16-byte aligned.
+ */
+#ifndef KMQ_H_
+#define KMQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  KMQ_OK = 0,
+  KMQ_ERR_NULL = 1,      /* a required pointer is NULL */
+  KMQ_ERR_BITS = 2,      /* bits is not 1, 2 or 4 */
+  KMQ_ERR_SHAPE = 3,     /* N, K or M out of range, or K not a multiple of 32/bits */
+  KMQ_ERR_ALIGN = 4,     /* a device pointer is not 16-byte aligned */
+  KMQ_ERR_WORKSPACE = 5, /* workspace missing or smaller than kmq_workspace_bytes() */
+  KMQ_ERR_LAYOUT = 6,    /* unknown layout id */
+  KMQ_ERR_CUDA = 7       /* the CUDA runtime reported an error (launch, copy) */
+} kmq_status;
+
+typedef enum {
+  KMQ_LAYOUT_CANONICAL = 0
+} kmq_layout;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int kmq_version(void);
+
+/* Static, NUL-terminated description of a status code. */
+const char* kmq_status_string(int status);
+
+/* Bytes of the packed index matrix, N * K * bits / 8; 0 if the arguments are invalid. */
+size_t kmq_packed_bytes(int64_t N, int64_t K, int bits, int layout);
+
+/* Bytes of scratch kmq_linear needs for this shape on the current device
+ * (fp32 partial sums of a split along K); may be 0. */
+size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M);
+
+/* Number of kernels one kmq_linear call launches for this shape (1 or 2), and
+ * a short static name of the kernel variant the dispatcher picks. */
+int kmq_linear_num_launches(int64_t N, int64_t K, int bits, int64_t M);
+const char* kmq_linear_variant(int64_t N, int64_t K, int bits, int64_t M);
+
+/*
+ * kmq_pack -- bit-pack centroid indices along K (the paper stores the
+ * quantised elements packed along the input dimension; Appendix
+ * "Benchmarking", "Kernel implementations").
+ *   idx    DEVICE uint8 [N, K] row-major; only the low `bits` bits are kept.
+ *   packed DEVICE uint32, kmq_packed_bytes() bytes, written in `layout`.
+ */
+kmq_status kmq_pack(const uint8_t* idx, int64_t N, int64_t K, int bits, int layout,
+                    uint32_t* packed, void* stream);
+
+/* kmq_unpack -- inverse of kmq_pack: idx DEVICE uint8 [N, K] is written. */
+kmq_status kmq_unpack(const uint32_t* packed, int64_t N, int64_t K, int bits, int layout,
+                      uint8_t* idx, void* stream);
+
+/*
+ * kmq_linear -- y[m,n] = sum_k x[m,k] * C_n[idx[n,k]], bf16 products
+ * accumulated in fp32, result rounded to bf16 (round-to-nearest-even).
+ * (Appendix "Benchmarking": Y^T = dequantize(W~) X^T; Appendix "Theoretical
+ * model of software-decoded formats": Y^T = W X^T with X, Y of shape m x h.)
+ *   packed    DEVICE uint32, canonical layout [N, K*bits/32].
+ *   codebooks DEVICE bf16 [N, 2^bits] row-major, C_n[i] at n*2^bits + i.
+ *   x         DEVICE bf16 [M, K] row-major.
+ *   y         DEVICE bf16 [M, N] row-major, fully overwritten.
+ *   workspace DEVICE, at least kmq_workspace_bytes(N,K,bits,M) bytes; may be
+ *             NULL when that is 0.  Contents on entry are ignored, contents on
+ *             return are unspecified.
+ * The order of the fp32 summation is fixed for a given shape and device, so
+ * repeated calls give bit-identical results.  Outputs for non-finite inputs
+ * are unspecified.
+ */
+kmq_status kmq_linear(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x,
+                      uint16_t* y, int64_t N, int64_t K, int bits, int64_t M, int layout,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * kmq_linear_host -- the same layer for a caller whose activations live in
+ * host memory: copies x (HOST bf16 [M,K]) into x_dev, runs kmq_linear, copies
+ * y_dev into y (HOST bf16 [M,N]) and synchronises `stream` before returning.
+ * The weights (packed, codebooks) stay resident on the device.
+ *   x_dev, y_dev  DEVICE staging buffers of M*K*2 and M*N*2 bytes.
+ */
+kmq_status kmq_linear_host(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x_host,
+                           uint16_t* y_host, int64_t N, int64_t K, int bits, int64_t M, int layout,
+                           uint16_t* x_dev, uint16_t* y_dev, void* workspace, size_t workspace_bytes,
+                           void* stream);
+
+/*
+ * kmq_dequant_to_bf16 -- materialise W^[n,k] = C_n[idx[n,k]] as a dense bf16
+ * matrix; every element is a bit-exact copy of a stored centroid.  This is
+ * the separate dequantise step the paper suggests ahead of a standard GEMM
+ * at large batch sizes and prefill (Appendix "Benchmarking", "Model
+ * benchmarks").
+ *   W  DEVICE bf16 [N, K] row-major, fully overwritten.
+ */
+kmq_status kmq_dequant_to_bf16(const uint32_t* packed, const uint16_t* codebooks, uint16_t* W,
+                               int64_t N, int64_t K, int bits, int layout, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KMQ_H_ */

@@ -1,0 +1,142 @@
+// extern "C" boundary of libkmq: argument validation and dispatch.
+#include <mutex>
+
+#include "kmq_common.cuh"
+
+namespace kmq {
+
+const DeviceInfo* device_info() {
+  constexpr int kMaxDevices = 64;
+  static DeviceInfo cache[kMaxDevices];
+  static bool valid[kMaxDevices] = {};
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!valid[dev]) {
+    int sms = 0, smem = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+    if (cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return nullptr;
+    cache[dev].sm_count = sms;
+    cache[dev].max_smem_optin = smem;
+    valid[dev] = true;
+  }
+  return &cache[dev];
+}
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+kmq_status check_shape(int64_t N, int64_t K, int bits, int64_t M) {
+  if (bits != 1 && bits != 2 && bits != 4) return KMQ_ERR_BITS;
+  const int64_t per = 32 / bits;
+  if (N < 1 || M < 1 || K < per || (K % per) != 0) return KMQ_ERR_SHAPE;
+  // keep every element count and byte offset inside int64 with room to spare
+  if (N > (int64_t(1) << 31) || K > (int64_t(1) << 31) || M > (int64_t(1) << 24)) return KMQ_ERR_SHAPE;
+  return KMQ_OK;
+}
+
+}  // namespace
+}  // namespace kmq
+
+using namespace kmq;
+
+extern "C" {
+
+int kmq_version(void) { return 100; }
+
+const char* kmq_status_string(int status) {
+  switch (status) {
+    case KMQ_OK: return "ok";
+    case KMQ_ERR_NULL: return "a required pointer is NULL";
+    case KMQ_ERR_BITS: return "bits must be 1, 2 or 4";
+    case KMQ_ERR_SHAPE: return "invalid shape (N, M >= 1; K a positive multiple of 32/bits)";
+    case KMQ_ERR_ALIGN: return "device pointers must be 16-byte aligned";
+    case KMQ_ERR_WORKSPACE: return "workspace missing or too small";
+    case KMQ_ERR_LAYOUT: return "unknown packed layout";
+    case KMQ_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+  }
+}
+
+size_t kmq_packed_bytes(int64_t N, int64_t K, int bits, int layout) {
+  if (layout != KMQ_LAYOUT_CANONICAL || check_shape(N, K, bits, 1) != KMQ_OK) return 0;
+  return (size_t)N * (size_t)(K / (32 / bits)) * 4u;
+}
+
+size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M) {
+  if (check_shape(N, K, bits, M) != KMQ_OK) return 0;
+  return plan_linear(N, K, bits, M).workspace;
+}
+
+int kmq_linear_num_launches(int64_t N, int64_t K, int bits, int64_t M) {
+  if (check_shape(N, K, bits, M) != KMQ_OK) return 0;
+  return plan_linear(N, K, bits, M).launches;
+}
+
+const char* kmq_linear_variant(int64_t N, int64_t K, int bits, int64_t M) {
+  if (check_shape(N, K, bits, M) != KMQ_OK) return "invalid";
+  return plan_linear(N, K, bits, M).name;
+}
+
+kmq_status kmq_pack(const uint8_t* idx, int64_t N, int64_t K, int bits, int layout, uint32_t* packed, void* stream) {
+  if (!idx || !packed) return KMQ_ERR_NULL;
+  if (kmq_status s = check_shape(N, K, bits, 1)) return s;
+  if (layout != KMQ_LAYOUT_CANONICAL) return KMQ_ERR_LAYOUT;
+  if (!aligned16(idx) || !aligned16(packed)) return KMQ_ERR_ALIGN;
+  return launch_pack(idx, N, K, bits, packed, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
+}
+
+kmq_status kmq_unpack(const uint32_t* packed, int64_t N, int64_t K, int bits, int layout, uint8_t* idx, void* stream) {
+  if (!idx || !packed) return KMQ_ERR_NULL;
+  if (kmq_status s = check_shape(N, K, bits, 1)) return s;
+  if (layout != KMQ_LAYOUT_CANONICAL) return KMQ_ERR_LAYOUT;
+  if (!aligned16(idx) || !aligned16(packed)) return KMQ_ERR_ALIGN;
+  return launch_unpack(packed, N, K, bits, idx, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
+}
+
+kmq_status kmq_linear(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x, uint16_t* y, int64_t N,
+                      int64_t K, int bits, int64_t M, int layout, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+  if (!packed || !codebooks || !x || !y) return KMQ_ERR_NULL;
+  if (kmq_status s = check_shape(N, K, bits, M)) return s;
+  if (layout != KMQ_LAYOUT_CANONICAL) return KMQ_ERR_LAYOUT;
+  if (!aligned16(packed) || !aligned16(codebooks) || !aligned16(x) || !aligned16(y)) return KMQ_ERR_ALIGN;
+  if (!device_info()) return KMQ_ERR_CUDA;
+  const LinearPlan plan = plan_linear(N, K, bits, M);
+  if (plan.workspace > 0) {
+    if (!workspace || workspace_bytes < plan.workspace) return KMQ_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return KMQ_ERR_ALIGN;
+  }
+  return launch_linear(plan, packed, codebooks, x, y, N, K, bits, M, workspace, (cudaStream_t)stream) == cudaSuccess
+             ? KMQ_OK
+             : KMQ_ERR_CUDA;
+}
+
+kmq_status kmq_linear_host(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x_host, uint16_t* y_host,
+                           int64_t N, int64_t K, int bits, int64_t M, int layout, uint16_t* x_dev, uint16_t* y_dev,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+  if (!x_host || !y_host || !x_dev || !y_dev) return KMQ_ERR_NULL;
+  if (!packed || !codebooks) return KMQ_ERR_NULL;
+  if (kmq_status s = check_shape(N, K, bits, M)) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return KMQ_ERR_CUDA;
+  if (kmq_status s = kmq_linear(packed, codebooks, x_dev, y_dev, N, K, bits, M, layout, workspace, workspace_bytes,
+                                stream))
+    return s;
+  if (cudaMemcpyAsync(y_host, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KMQ_ERR_CUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
+}
+
+kmq_status kmq_dequant_to_bf16(const uint32_t* packed, const uint16_t* codebooks, uint16_t* W, int64_t N, int64_t K,
+                               int bits, int layout, void* stream) {
+  if (!packed || !codebooks || !W) return KMQ_ERR_NULL;
+  if (kmq_status s = check_shape(N, K, bits, 1)) return s;
+  if (layout != KMQ_LAYOUT_CANONICAL) return KMQ_ERR_LAYOUT;
+  if (!aligned16(packed) || !aligned16(codebooks) || !aligned16(W)) return KMQ_ERR_ALIGN;
+  return launch_dequant(packed, codebooks, W, N, K, bits, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK
+                                                                                               : KMQ_ERR_CUDA;
+}
+
+}  // extern "C"

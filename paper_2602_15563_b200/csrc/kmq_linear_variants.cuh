@@ -1,0 +1,14 @@
+// Kernel variants behind kmq_linear and their launchers.
+#pragma once
+#include "kmq_common.cuh"
+
+namespace kmq {
+
+enum LinearVariant : int {
+  kVariantGeneric = 0,
+};
+
+cudaError_t launch_linear_generic(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                                  int64_t K, int bits, int64_t M, cudaStream_t s);
+
+}  // namespace kmq

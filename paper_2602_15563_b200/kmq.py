@@ -1,0 +1,148 @@
+"""ctypes binding of libkmq: same names as the C entry points, argument
+marshalling only.  Every step of the layer runs in the CUDA library; there is
+no Python or CPU implementation behind these calls, and loading fails loudly
+when the shared library has not been built.
+
+Tensor arguments are ``torch`` CUDA tensors (used for device memory only) or
+raw integer device addresses; ``stream`` defaults to torch's current stream.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libkmq.so")
+_lib = None
+
+KMQ_OK = 0
+KMQ_ERR_NULL, KMQ_ERR_BITS, KMQ_ERR_SHAPE, KMQ_ERR_ALIGN = 1, 2, 3, 4
+KMQ_ERR_WORKSPACE, KMQ_ERR_LAYOUT, KMQ_ERR_CUDA = 5, 6, 7
+KMQ_LAYOUT_CANONICAL = 0
+
+_i64, _int, _ptr, _sz = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t
+
+# name -> (restype, argtypes); mirrors include/kmq.h
+SIGNATURES = {
+    "kmq_version": (_int, []),
+    "kmq_status_string": (ctypes.c_char_p, [_int]),
+    "kmq_packed_bytes": (_sz, [_i64, _i64, _int, _int]),
+    "kmq_workspace_bytes": (_sz, [_i64, _i64, _int, _i64]),
+    "kmq_linear_num_launches": (_int, [_i64, _i64, _int, _i64]),
+    "kmq_linear_variant": (ctypes.c_char_p, [_i64, _i64, _int, _i64]),
+    "kmq_pack": (_int, [_ptr, _i64, _i64, _int, _int, _ptr, _ptr]),
+    "kmq_unpack": (_int, [_ptr, _i64, _i64, _int, _int, _ptr, _ptr]),
+    "kmq_linear": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr, _sz, _ptr]),
+    "kmq_linear_host": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr, _ptr, _ptr, _sz, _ptr]),
+    "kmq_dequant_to_bf16": (_int, [_ptr, _ptr, _ptr, _i64, _i64, _int, _int, _ptr]),
+}
+
+
+class KmqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libkmq.so (once).  Raises if it is missing: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(
+                f"{_LIB_PATH} not found: build it with "
+                "`python -m paper_2602_15563_b200.build` (needs nvcc); libkmq has no CPU fallback")
+        handle = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def _addr(t) -> int:
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(status: int, where: str) -> None:
+    if status != KMQ_OK:
+        raise KmqError(status, where)
+
+
+def status_string(status: int) -> str:
+    return lib().kmq_status_string(int(status)).decode()
+
+
+def kmq_version() -> int:
+    return lib().kmq_version()
+
+
+def kmq_packed_bytes(N, K, bits, layout=KMQ_LAYOUT_CANONICAL) -> int:
+    return lib().kmq_packed_bytes(N, K, bits, layout)
+
+
+def kmq_workspace_bytes(N, K, bits, M) -> int:
+    return lib().kmq_workspace_bytes(N, K, bits, M)
+
+
+def kmq_linear_num_launches(N, K, bits, M) -> int:
+    return lib().kmq_linear_num_launches(N, K, bits, M)
+
+
+def kmq_linear_variant(N, K, bits, M) -> str:
+    return lib().kmq_linear_variant(N, K, bits, M).decode()
+
+
+def kmq_pack(idx, N, K, bits, packed, layout=KMQ_LAYOUT_CANONICAL, stream=None, check=True) -> int:
+    st = lib().kmq_pack(_addr(idx), N, K, bits, layout, _addr(packed), _stream(stream))
+    if check:
+        _check(st, "kmq_pack")
+    return st
+
+
+def kmq_unpack(packed, N, K, bits, idx, layout=KMQ_LAYOUT_CANONICAL, stream=None, check=True) -> int:
+    st = lib().kmq_unpack(_addr(packed), N, K, bits, layout, _addr(idx), _stream(stream))
+    if check:
+        _check(st, "kmq_unpack")
+    return st
+
+
+def kmq_linear(packed, codebooks, x, y, N, K, bits, M, workspace=None, workspace_bytes=None,
+               layout=KMQ_LAYOUT_CANONICAL, stream=None, check=True) -> int:
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None or isinstance(workspace, int) else workspace.numel() * workspace.element_size()
+    st = lib().kmq_linear(_addr(packed), _addr(codebooks), _addr(x), _addr(y), N, K, bits, M, layout,
+                          _addr(workspace), workspace_bytes, _stream(stream))
+    if check:
+        _check(st, "kmq_linear")
+    return st
+
+
+def kmq_linear_host(packed, codebooks, x_host, y_host, N, K, bits, M, x_dev, y_dev, workspace=None,
+                    workspace_bytes=None, layout=KMQ_LAYOUT_CANONICAL, stream=None, check=True) -> int:
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None or isinstance(workspace, int) else workspace.numel() * workspace.element_size()
+    st = lib().kmq_linear_host(_addr(packed), _addr(codebooks), _addr(x_host), _addr(y_host), N, K, bits, M, layout,
+                               _addr(x_dev), _addr(y_dev), _addr(workspace), workspace_bytes, _stream(stream))
+    if check:
+        _check(st, "kmq_linear_host")
+    return st
+
+
+def kmq_dequant_to_bf16(packed, codebooks, W, N, K, bits, layout=KMQ_LAYOUT_CANONICAL, stream=None, check=True) -> int:
+    st = lib().kmq_dequant_to_bf16(_addr(packed), _addr(codebooks), _addr(W), N, K, bits, layout, _stream(stream))
+    if check:
+        _check(st, "kmq_dequant_to_bf16")
+    return st

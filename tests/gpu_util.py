@@ -1,0 +1,63 @@
+"""Helpers shared by the GPU parity tests: move a synthetic layer to the device,
+run the library through its C ABI, bring the results back as NumPy arrays."""
+import numpy as np
+import torch
+
+from paper_2602_15563_b200 import kmq
+
+CANARY = 0x5A
+
+
+def dev_bytes(nbytes: int, pad: int = 256):
+    """A device buffer of `nbytes` with canary bands on both sides.
+    Returns (whole uint8 tensor, offset of the payload)."""
+    total = nbytes + 2 * pad
+    buf = torch.full((total,), CANARY, dtype=torch.uint8, device="cuda")
+    return buf, pad
+
+
+def canaries_intact(buf: torch.Tensor, off: int, nbytes: int) -> bool:
+    head = buf[:off]
+    tail = buf[off + nbytes:]
+    return bool((head == CANARY).all().item() and (tail == CANARY).all().item())
+
+
+def to_dev_u16(a: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda()
+
+
+def gpu_pack(idx: np.ndarray, bits: int) -> torch.Tensor:
+    N, K = idx.shape
+    d_idx = torch.from_numpy(np.ascontiguousarray(idx)).cuda()
+    packed = torch.empty(kmq.kmq_packed_bytes(N, K, bits) // 4, dtype=torch.int32, device="cuda")
+    kmq.kmq_pack(d_idx, N, K, bits, packed)
+    return packed
+
+
+def packed_to_numpy(packed: torch.Tensor, N: int) -> np.ndarray:
+    return packed.cpu().numpy().view(np.uint32).reshape(N, -1)
+
+
+def gpu_dequant(packed: torch.Tensor, cb: np.ndarray, N: int, K: int, bits: int) -> np.ndarray:
+    d_cb = to_dev_u16(cb)
+    nbytes = N * K * 2
+    buf, off = dev_bytes(nbytes)
+    kmq.kmq_dequant_to_bf16(packed, d_cb, buf.data_ptr() + off, N, K, bits)
+    torch.cuda.synchronize()
+    assert canaries_intact(buf, off, nbytes), "dequant wrote outside W"
+    return buf[off:off + nbytes].cpu().numpy().view(np.uint16).reshape(N, K)
+
+
+def gpu_linear(packed: torch.Tensor, cb: np.ndarray, x: np.ndarray, N: int, K: int, bits: int) -> np.ndarray:
+    M = x.shape[0]
+    d_cb, d_x = to_dev_u16(cb), to_dev_u16(x)
+    nbytes = M * N * 2
+    buf, off = dev_bytes(nbytes)
+    ws_bytes = kmq.kmq_workspace_bytes(N, K, bits, M)
+    wsbuf, wsoff = dev_bytes(max(ws_bytes, 16))
+    kmq.kmq_linear(packed, d_cb, d_x, buf.data_ptr() + off, N, K, bits, M,
+                   wsbuf.data_ptr() + wsoff, ws_bytes)
+    torch.cuda.synchronize()
+    assert canaries_intact(buf, off, nbytes), "linear wrote outside y"
+    assert canaries_intact(wsbuf, wsoff, max(ws_bytes, 16)), "linear wrote outside its workspace"
+    return buf[off:off + nbytes].cpu().numpy().view(np.uint16).reshape(M, N)
