@@ -5,13 +5,18 @@
 namespace kmq {
 
 LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M) {
-  (void)N; (void)K; (void)bits; (void)M;
   LinearPlan p;
-  p.variant = kVariantGeneric;
-  p.launches = 1;
   p.workspace = 0;
   p.split_k = 1;
-  p.name = "generic_warp_per_row";
+  if (linear_mma_supports(N, K, bits, M)) {
+    p.variant = kVariantMma;
+    p.launches = (int)((M + 7) / 8);
+    p.name = bits == 1 ? "mma_sign_b1" : bits == 2 ? "mma_prmt_b2" : "mma_pairtable_b4";
+  } else {
+    p.variant = kVariantGeneric;
+    p.launches = 1;
+    p.name = "generic_warp_per_row";
+  }
   return p;
 }
 
@@ -19,6 +24,8 @@ cudaError_t launch_linear(const LinearPlan& plan, const uint32_t* packed, const 
                           uint16_t* y, int64_t N, int64_t K, int bits, int64_t M, void* workspace, cudaStream_t s) {
   (void)workspace;
   switch (plan.variant) {
+    case kVariantMma:
+      return launch_linear_mma(packed, cb, x, y, N, K, bits, M, s);
     case kVariantGeneric:
     default:
       return launch_linear_generic(packed, cb, x, y, N, K, bits, M, s);

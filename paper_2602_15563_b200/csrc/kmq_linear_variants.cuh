@@ -5,10 +5,15 @@
 namespace kmq {
 
 enum LinearVariant : int {
-  kVariantGeneric = 0,
+  kVariantGeneric = 0,   // any legal shape, CUDA-core FMAs, one warp per output row
+  kVariantMma = 1,       // K*bits % 128 == 0: tensor-core GEMV, 8 batch rows per launch
 };
 
 cudaError_t launch_linear_generic(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                   int64_t K, int bits, int64_t M, cudaStream_t s);
+
+bool linear_mma_supports(int64_t N, int64_t K, int bits, int64_t M);
+cudaError_t launch_linear_mma(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                              int64_t K, int bits, int64_t M, cudaStream_t s);
 
 }  // namespace kmq
