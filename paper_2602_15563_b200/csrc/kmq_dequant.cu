@@ -7,30 +7,39 @@
 namespace kmq {
 namespace {
 
-template <int BITS>
-__device__ __forceinline__ uint32_t load_chunk_bits(const uint32_t* __restrict__ packed, int64_t row_word0, int64_t c) {
-  if constexpr (BITS == 4) {
-    return __ldg(packed + row_word0 + c);
+// The 8*BITS bits that hold weights 8c .. 8c+7 of row n, fields LSB first.
+template <int BITS, bool TUNED>
+__device__ __forceinline__ uint32_t load_chunk_bits(const uint32_t* __restrict__ packed, int64_t n, int64_t wpr,
+                                                    int64_t steps, int64_t c) {
+  if constexpr (TUNED) {
+    // the fields of a chunk are spread over its word: permute the word back, then cut the chunk out
+    constexpr int CPW = 4 / BITS;   // 8-weight chunks per word
+    const uint32_t w = canonical_from_tuned<BITS>(__ldg(packed + tuned_word_index(n, c / CPW, steps)));
+    if constexpr (BITS == 4) return w;
+    return (w >> ((int)(c % CPW) * 8 * BITS)) & ((1u << (8 * BITS)) - 1u);
+  } else if constexpr (BITS == 4) {
+    return __ldg(packed + n * wpr + c);
   } else if constexpr (BITS == 2) {
-    return __ldg(reinterpret_cast<const uint16_t*>(packed + row_word0) + c);
+    return __ldg(reinterpret_cast<const uint16_t*>(packed + n * wpr) + c);
   } else {
-    return __ldg(reinterpret_cast<const uint8_t*>(packed + row_word0) + c);
+    return __ldg(reinterpret_cast<const uint8_t*>(packed + n * wpr) + c);
   }
 }
 
-template <int BITS>
+template <int BITS, bool TUNED>
 __global__ void __launch_bounds__(256) dequant_kernel(const uint32_t* __restrict__ packed,
                                                       const uint16_t* __restrict__ cb, uint16_t* __restrict__ W,
                                                       int64_t N, int64_t K) {
   constexpr int Q = 1 << BITS;
   const int64_t cpr = K >> 3;            // 8-weight chunks per row
   const int64_t wpr = K / (32 / BITS);   // words per row
+  const int64_t steps = tuned_steps(wpr);
   const int64_t total = N * cpr;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t chunk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; chunk < total; chunk += stride) {
     const int64_t n = chunk / cpr;
     const int64_t c = chunk - n * cpr;
-    const uint32_t v = load_chunk_bits<BITS>(packed, n * wpr, c);
+    const uint32_t v = load_chunk_bits<BITS, TUNED>(packed, n, wpr, steps, c);
     uint32_t o[4];
     if constexpr (BITS == 1) {
       // codebook = 4 bytes {c0, c1}; a selector nibble pair picks bytes (2i, 2i+1)
@@ -63,7 +72,7 @@ __global__ void __launch_bounds__(256) dequant_kernel(const uint32_t* __restrict
 }  // namespace
 
 cudaError_t launch_dequant(const uint32_t* packed, const uint16_t* cb, uint16_t* W, int64_t N, int64_t K, int bits,
-                           cudaStream_t s) {
+                           int layout, cudaStream_t s) {
   const DeviceInfo* di = device_info();
   if (!di) return cudaGetLastError();
   const int64_t total = N * (K >> 3);
@@ -71,9 +80,13 @@ cudaError_t launch_dequant(const uint32_t* packed, const uint16_t* cb, uint16_t*
   const int64_t cap = (int64_t)di->sm_count * 32;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  if (bits == 1) dequant_kernel<1><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
-  else if (bits == 2) dequant_kernel<2><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
-  else dequant_kernel<4><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  const bool tuned = layout == KMQ_LAYOUT_TUNED;
+  if (bits == 1 && tuned) dequant_kernel<1, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  else if (bits == 1) dequant_kernel<1, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  else if (bits == 2 && tuned) dequant_kernel<2, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  else if (bits == 2) dequant_kernel<2, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  else if (tuned) dequant_kernel<4, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  else dequant_kernel<4, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
   return cudaGetLastError();
 }
 

@@ -1,4 +1,4 @@
-// kmq_linear for batch rows M <= 8 per pass: one CTA per 16 output rows, the
+// kmq_linear on the canonical packed layout, batch rows M <= 8 per pass: one CTA per 16 output rows, the
 // warps of the CTA split K, every warp streams its slices of the packed rows
 // with 128-bit loads (several in flight per lane), rebuilds the bf16 weights
 // in registers directly in the operand layout of mma.sync.m16n8k16 (weights
@@ -22,6 +22,7 @@
 // same order, so the canonical packed layout is consumed as is.
 #include "kmq_common.cuh"
 #include "kmq_linear_variants.cuh"
+#include "kmq_mma_common.cuh"
 
 namespace kmq {
 namespace {
@@ -46,20 +47,6 @@ struct Geo {
 template <int BITS, int MMAX>
 constexpr int smem_bytes() {
   return Geo<BITS>::kTableBytes + kWarps * MMAX * Geo<BITS>::kRowStride + kRedBytes + 16 * kWarps * 4;
-}
-
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-  uint32_t d;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-  return d;
 }
 
 // ---------------------------------------------------------------------------
@@ -124,23 +111,6 @@ __device__ __forceinline__ void stage_step(const uint16_t* __restrict__ x, int64
   for (int m = lane >> 4; m < M; m += 2)
     stage_block<BITS>(x + (int64_t)m * K, k0, in_k, xs_warp + m * G::kRowStride + j * G::kMmaPerWord * 32 + t * 8);
 }
-
-// b = 2: byte tables {lo bytes of c0..c3}, {hi bytes of c0..c3} of one row
-struct Dec2 {
-  uint32_t lo, hi;
-  __device__ __forceinline__ void init(const uint16_t* __restrict__ cb_row) {
-    const uint2 c = __ldg(reinterpret_cast<const uint2*>(cb_row));
-    lo = prmt(c.x, c.y, 0x6420u);
-    hi = prmt(c.x, c.y, 0x7531u);
-  }
-  // phase q of a word: fields q, q+4, q+8, q+12 -> (W_q, W_q+4) and (W_q+8, W_q+12)
-  __device__ __forceinline__ void pair(uint32_t w, int q, uint32_t& a_first, uint32_t& a_second) const {
-    const uint32_t f = (w >> (2 * q)) & 0x03030303u;
-    const uint32_t sel = f * 0x11u + 0x40404040u;   // per byte: nibbles (i, 4 + i) select (lo_i, hi_i)
-    a_first = prmt(lo, hi, sel);
-    a_second = prmt(lo, hi, sel >> 16);
-  }
-};
 
 template <int BITS, int MMAX>
 __global__ void __launch_bounds__(kThreads) linear_mma_kernel(const uint32_t* __restrict__ packed,
