@@ -24,9 +24,25 @@
  *   - bf16 values are passed as uint16_t bit patterns.
  *   - Shapes: N output rows, K input features, M batch rows.  N, M >= 1;
  *     K >= 32/bits and K % (32/bits) == 0.  Buffers must not overlap.
- *   - Canonical packed layout (KMQ_LAYOUT_CANONICAL): row-major
- *     uint32 [N, K*bits/32]; bits [i*bits, (i+1)*bits) of word j of row n hold
- *     idx[n, j*(32/bits) + i] (fields LSB first, packed along K).
+ *   - Packed layouts.  With wpr = K*bits/32 words per row, word j of row n
+ *     holds the 32/bits indices idx[n, j*(32/bits) + i], i = 0..32/bits-1.
+ *     KMQ_LAYOUT_CANONICAL (the interchange format): row-major uint32 [N, wpr],
+ *     field i of a word at bits [i*bits, (i+1)*bits), fields LSB first.
+ *     KMQ_LAYOUT_TUNED (what the fast kernels read; the paper names an
+ *     "optimized data layout" as the way to reach bandwidth, Appendix
+ *     "Benchmarking", "Micro-benchmarks"): tile-major.  Rows are grouped in
+ *     tiles of 16 and the words of a row in steps of 16; with steps =
+ *     ceil(wpr/16), word (n, j) is stored at word index
+ *       (((n/16)*steps + j/16)*16 + n%16)*16 + j%16,
+ *     so one step of one tile is a contiguous 1 KB block; rows beyond N and
+ *     words beyond wpr are zero padding (kmq_packed_bytes gives the padded
+ *     size).  Inside a word the fields sit where the tensor-core kernels can
+ *     extract four consecutive weights with the fewest integer instructions:
+ *       bits = 4: field i at bits [4i, 4i+4) (as canonical);
+ *       bits = 2: field i = 4p + c (p, c in 0..3) at bits [2p + 8c, 2p + 8c + 2);
+ *       bits = 1: field i = 2c at bit 15 - c, field i = 2c + 1 at bit 31 - c.
+ *     Every entry point accepts either layout; kmq_pack writes the one asked
+ *     for, the others must be told which one `packed` is in.
  *   - All device pointers must be 16-byte aligned.
  */
 #ifndef KMQ_H_
@@ -51,7 +67,8 @@ typedef enum {
 } kmq_status;
 
 typedef enum {
-  KMQ_LAYOUT_CANONICAL = 0
+  KMQ_LAYOUT_CANONICAL = 0,
+  KMQ_LAYOUT_TUNED = 1
 } kmq_layout;
 
 /* Library version (major*10000 + minor*100 + patch). */
@@ -60,17 +77,18 @@ int kmq_version(void);
 /* Static, NUL-terminated description of a status code. */
 const char* kmq_status_string(int status);
 
-/* Bytes of the packed index matrix, N * K * bits / 8; 0 if the arguments are invalid. */
+/* Bytes of the packed index matrix: N * K * bits / 8 (canonical) or the padded
+ * tile-major size (tuned); 0 if the arguments are invalid. */
 size_t kmq_packed_bytes(int64_t N, int64_t K, int bits, int layout);
 
 /* Bytes of scratch kmq_linear needs for this shape on the current device
  * (fp32 partial sums of a split along K); may be 0. */
-size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M);
+size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M, int layout);
 
 /* Number of kernels one kmq_linear call launches for this shape (1 or 2), and
  * a short static name of the kernel variant the dispatcher picks. */
-int kmq_linear_num_launches(int64_t N, int64_t K, int bits, int64_t M);
-const char* kmq_linear_variant(int64_t N, int64_t K, int bits, int64_t M);
+int kmq_linear_num_launches(int64_t N, int64_t K, int bits, int64_t M, int layout);
+const char* kmq_linear_variant(int64_t N, int64_t K, int bits, int64_t M, int layout);
 
 /*
  * kmq_pack -- bit-pack centroid indices along K (the paper stores the
@@ -91,11 +109,11 @@ kmq_status kmq_unpack(const uint32_t* packed, int64_t N, int64_t K, int bits, in
  * accumulated in fp32, result rounded to bf16 (round-to-nearest-even).
  * (Appendix "Benchmarking": Y^T = dequantize(W~) X^T; Appendix "Theoretical
  * model of software-decoded formats": Y^T = W X^T with X, Y of shape m x h.)
- *   packed    DEVICE uint32, canonical layout [N, K*bits/32].
+ *   packed    DEVICE uint32, kmq_packed_bytes() bytes, in `layout`.
  *   codebooks DEVICE bf16 [N, 2^bits] row-major, C_n[i] at n*2^bits + i.
  *   x         DEVICE bf16 [M, K] row-major.
  *   y         DEVICE bf16 [M, N] row-major, fully overwritten.
- *   workspace DEVICE, at least kmq_workspace_bytes(N,K,bits,M) bytes; may be
+ *   workspace DEVICE, at least kmq_workspace_bytes(N,K,bits,M,layout) bytes; may be
  *             NULL when that is 0.  Contents on entry are ignored, contents on
  *             return are unspecified.
  * The order of the fp32 summation is fixed for a given shape and device, so

@@ -27,6 +27,7 @@ const DeviceInfo* device_info() {
 namespace {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool known_layout(int layout) { return layout == KMQ_LAYOUT_CANONICAL || layout == KMQ_LAYOUT_TUNED; }
 
 kmq_status check_shape(int64_t N, int64_t K, int bits, int64_t M) {
   if (bits != 1 && bits != 2 && bits != 4) return KMQ_ERR_BITS;
@@ -61,39 +62,41 @@ const char* kmq_status_string(int status) {
 }
 
 size_t kmq_packed_bytes(int64_t N, int64_t K, int bits, int layout) {
-  if (layout != KMQ_LAYOUT_CANONICAL || check_shape(N, K, bits, 1) != KMQ_OK) return 0;
-  return (size_t)N * (size_t)(K / (32 / bits)) * 4u;
+  if (!known_layout(layout) || check_shape(N, K, bits, 1) != KMQ_OK) return 0;
+  const int64_t wpr = K / (32 / bits);
+  if (layout == KMQ_LAYOUT_TUNED) return (size_t)tuned_total_words(N, wpr) * 4u;
+  return (size_t)N * (size_t)wpr * 4u;
 }
 
-size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M) {
-  if (check_shape(N, K, bits, M) != KMQ_OK) return 0;
-  return plan_linear(N, K, bits, M).workspace;
+size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M, int layout) {
+  if (!known_layout(layout) || check_shape(N, K, bits, M) != KMQ_OK) return 0;
+  return plan_linear(N, K, bits, M, layout).workspace;
 }
 
-int kmq_linear_num_launches(int64_t N, int64_t K, int bits, int64_t M) {
-  if (check_shape(N, K, bits, M) != KMQ_OK) return 0;
-  return plan_linear(N, K, bits, M).launches;
+int kmq_linear_num_launches(int64_t N, int64_t K, int bits, int64_t M, int layout) {
+  if (!known_layout(layout) || check_shape(N, K, bits, M) != KMQ_OK) return 0;
+  return plan_linear(N, K, bits, M, layout).launches;
 }
 
-const char* kmq_linear_variant(int64_t N, int64_t K, int bits, int64_t M) {
-  if (check_shape(N, K, bits, M) != KMQ_OK) return "invalid";
-  return plan_linear(N, K, bits, M).name;
+const char* kmq_linear_variant(int64_t N, int64_t K, int bits, int64_t M, int layout) {
+  if (!known_layout(layout) || check_shape(N, K, bits, M) != KMQ_OK) return "invalid";
+  return plan_linear(N, K, bits, M, layout).name;
 }
 
 kmq_status kmq_pack(const uint8_t* idx, int64_t N, int64_t K, int bits, int layout, uint32_t* packed, void* stream) {
   if (!idx || !packed) return KMQ_ERR_NULL;
   if (kmq_status s = check_shape(N, K, bits, 1)) return s;
-  if (layout != KMQ_LAYOUT_CANONICAL) return KMQ_ERR_LAYOUT;
+  if (!known_layout(layout)) return KMQ_ERR_LAYOUT;
   if (!aligned16(idx) || !aligned16(packed)) return KMQ_ERR_ALIGN;
-  return launch_pack(idx, N, K, bits, packed, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
+  return launch_pack(idx, N, K, bits, layout, packed, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
 }
 
 kmq_status kmq_unpack(const uint32_t* packed, int64_t N, int64_t K, int bits, int layout, uint8_t* idx, void* stream) {
   if (!idx || !packed) return KMQ_ERR_NULL;
   if (kmq_status s = check_shape(N, K, bits, 1)) return s;
-  if (layout != KMQ_LAYOUT_CANONICAL) return KMQ_ERR_LAYOUT;
+  if (!known_layout(layout)) return KMQ_ERR_LAYOUT;
   if (!aligned16(idx) || !aligned16(packed)) return KMQ_ERR_ALIGN;
-  return launch_unpack(packed, N, K, bits, idx, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
+  return launch_unpack(packed, N, K, bits, layout, idx, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
 }
 
 kmq_status kmq_linear(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x, uint16_t* y, int64_t N,
@@ -101,15 +104,16 @@ kmq_status kmq_linear(const uint32_t* packed, const uint16_t* codebooks, const u
                       void* stream) {
   if (!packed || !codebooks || !x || !y) return KMQ_ERR_NULL;
   if (kmq_status s = check_shape(N, K, bits, M)) return s;
-  if (layout != KMQ_LAYOUT_CANONICAL) return KMQ_ERR_LAYOUT;
+  if (!known_layout(layout)) return KMQ_ERR_LAYOUT;
   if (!aligned16(packed) || !aligned16(codebooks) || !aligned16(x) || !aligned16(y)) return KMQ_ERR_ALIGN;
   if (!device_info()) return KMQ_ERR_CUDA;
-  const LinearPlan plan = plan_linear(N, K, bits, M);
+  const LinearPlan plan = plan_linear(N, K, bits, M, layout);
   if (plan.workspace > 0) {
     if (!workspace || workspace_bytes < plan.workspace) return KMQ_ERR_WORKSPACE;
     if (!aligned16(workspace)) return KMQ_ERR_ALIGN;
   }
-  return launch_linear(plan, packed, codebooks, x, y, N, K, bits, M, workspace, (cudaStream_t)stream) == cudaSuccess
+  return launch_linear(plan, packed, codebooks, x, y, N, K, bits, M, layout, workspace, (cudaStream_t)stream) ==
+                 cudaSuccess
              ? KMQ_OK
              : KMQ_ERR_CUDA;
 }
@@ -133,9 +137,9 @@ kmq_status kmq_dequant_to_bf16(const uint32_t* packed, const uint16_t* codebooks
                                int bits, int layout, void* stream) {
   if (!packed || !codebooks || !W) return KMQ_ERR_NULL;
   if (kmq_status s = check_shape(N, K, bits, 1)) return s;
-  if (layout != KMQ_LAYOUT_CANONICAL) return KMQ_ERR_LAYOUT;
+  if (!known_layout(layout)) return KMQ_ERR_LAYOUT;
   if (!aligned16(packed) || !aligned16(codebooks) || !aligned16(W)) return KMQ_ERR_ALIGN;
-  return launch_dequant(packed, codebooks, W, N, K, bits, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK
+  return launch_dequant(packed, codebooks, W, N, K, bits, layout, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK
                                                                                                : KMQ_ERR_CUDA;
 }
 

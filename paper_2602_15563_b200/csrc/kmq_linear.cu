@@ -1,17 +1,20 @@
-// Host-side dispatch of kmq_linear: picks a kernel variant for (bits, M, N, K).
+// Host-side dispatch of kmq_linear: picks a kernel variant for (bits, M, N, K, layout).
 #include "kmq_common.cuh"
 #include "kmq_linear_variants.cuh"
 
 namespace kmq {
 
-LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M) {
+LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
   LinearPlan p;
   p.workspace = 0;
   p.split_k = 1;
   if (linear_mma_supports(N, K, bits, M)) {
-    p.variant = kVariantMma;
+    const bool tuned = layout == KMQ_LAYOUT_TUNED;
+    p.variant = tuned ? kVariantTiled : kVariantMma;
     p.launches = (int)((M + 7) / 8);
-    p.name = bits == 1 ? "mma_sign_b1" : bits == 2 ? "mma_prmt_b2" : "mma_pairtable_b4";
+    if (bits == 4) p.name = tuned ? "tiled_pairtable_b4" : "staged_pairtable_b4";
+    else if (bits == 2) p.name = tuned ? "tiled_prmt_b2" : "staged_prmt_b2";
+    else p.name = tuned ? "tiled_sign_b1" : "staged_sign_b1";
   } else {
     p.variant = kVariantGeneric;
     p.launches = 1;
@@ -21,14 +24,17 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M) {
 }
 
 cudaError_t launch_linear(const LinearPlan& plan, const uint32_t* packed, const uint16_t* cb, const uint16_t* x,
-                          uint16_t* y, int64_t N, int64_t K, int bits, int64_t M, void* workspace, cudaStream_t s) {
+                          uint16_t* y, int64_t N, int64_t K, int bits, int64_t M, int layout, void* workspace,
+                          cudaStream_t s) {
   (void)workspace;
   switch (plan.variant) {
+    case kVariantTiled:
+      return launch_linear_tiled(packed, cb, x, y, N, K, bits, M, s);
     case kVariantMma:
       return launch_linear_mma(packed, cb, x, y, N, K, bits, M, s);
     case kVariantGeneric:
     default:
-      return launch_linear_generic(packed, cb, x, y, N, K, bits, M, s);
+      return launch_linear_generic(packed, cb, x, y, N, K, bits, M, layout, s);
   }
 }
 

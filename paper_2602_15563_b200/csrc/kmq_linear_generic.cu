@@ -8,7 +8,7 @@ namespace {
 
 constexpr int kWarpsPerCta = 8;
 
-template <int BITS, int MB>
+template <int BITS, int MB, bool TUNED>
 __global__ void __launch_bounds__(kWarpsPerCta * 32) linear_generic_kernel(
     const uint32_t* __restrict__ packed, const uint16_t* __restrict__ cb, const uint16_t* __restrict__ x,
     uint16_t* __restrict__ y, int64_t N, int64_t K, int64_t M) {
@@ -24,13 +24,15 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) linear_generic_kernel(
   __syncwarp();
 
   const int64_t wpr = K / PER;
-  const uint32_t* row = packed + n * wpr;
+  const uint32_t* row = packed + n * wpr;   // canonical layout only
+  const int64_t steps = tuned_steps(wpr);
   for (int64_t m0 = 0; m0 < M; m0 += MB) {
     float acc[MB];
 #pragma unroll
     for (int mm = 0; mm < MB; ++mm) acc[mm] = 0.f;
     for (int64_t j = lane; j < wpr; j += 32) {
-      const uint32_t word = __ldg(row + j);
+      const uint32_t word =
+          TUNED ? canonical_from_tuned<BITS>(__ldg(packed + tuned_word_index(n, j, steps))) : __ldg(row + j);
 #pragma unroll
       for (int q = 0; q < PER / 8; ++q) {
         float wv[8];
@@ -63,12 +65,16 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) linear_generic_kernel(
 }  // namespace
 
 cudaError_t launch_linear_generic(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
-                                  int64_t K, int bits, int64_t M, cudaStream_t s) {
+                                  int64_t K, int bits, int64_t M, int layout, cudaStream_t s) {
   const unsigned grid = (unsigned)((N + kWarpsPerCta - 1) / kWarpsPerCta);
   const int threads = kWarpsPerCta * 32;
-  if (bits == 1) linear_generic_kernel<1, 4><<<grid, threads, 0, s>>>(packed, cb, x, y, N, K, M);
-  else if (bits == 2) linear_generic_kernel<2, 4><<<grid, threads, 0, s>>>(packed, cb, x, y, N, K, M);
-  else linear_generic_kernel<4, 4><<<grid, threads, 0, s>>>(packed, cb, x, y, N, K, M);
+  const bool tuned = layout == KMQ_LAYOUT_TUNED;
+  if (bits == 1 && tuned) linear_generic_kernel<1, 4, true><<<grid, threads, 0, s>>>(packed, cb, x, y, N, K, M);
+  else if (bits == 1) linear_generic_kernel<1, 4, false><<<grid, threads, 0, s>>>(packed, cb, x, y, N, K, M);
+  else if (bits == 2 && tuned) linear_generic_kernel<2, 4, true><<<grid, threads, 0, s>>>(packed, cb, x, y, N, K, M);
+  else if (bits == 2) linear_generic_kernel<2, 4, false><<<grid, threads, 0, s>>>(packed, cb, x, y, N, K, M);
+  else if (tuned) linear_generic_kernel<4, 4, true><<<grid, threads, 0, s>>>(packed, cb, x, y, N, K, M);
+  else linear_generic_kernel<4, 4, false><<<grid, threads, 0, s>>>(packed, cb, x, y, N, K, M);
   return cudaGetLastError();
 }
 

@@ -311,7 +311,7 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
 
 bool linear_mma_supports(int64_t N, int64_t K, int bits, int64_t M) {
   (void)M;
-  return (K * bits) % 128 == 0 && (N + kRows - 1) / kRows <= 0x7FFFFFFF;
+  return (K * bits) % 128 == 0 && K <= (int64_t(1) << 30) && (N + kRows - 1) / kRows <= 0x7FFFFFFF;
 }
 
 // Batches larger than 8 are processed 8 rows at a time (one launch each).

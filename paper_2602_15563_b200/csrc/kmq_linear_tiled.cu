@@ -1,0 +1,309 @@
+// kmq_linear on the tuned (tile-major) packed layout, batch rows M <= 8 per pass.
+//
+// One CTA owns one tile of 16 output rows; its 8 warps split K step by step (a step = 64 packed bytes of each
+// row = 1 KB of the tile, stored contiguously).  Per step a warp
+//   - has the step's 1 KB of packed indices in registers: two 512-byte coalesced 128-bit loads issued several
+//     steps earlier (a ring of kStages steps per warp),
+//   - copies the activations under the step into its own slice of shared memory (prefetched into registers
+//     together with the weights), so that the B fragments are conflict-free 16-byte shared loads,
+//   - rebuilds the bf16 weights in registers in the A-operand layout of mma.sync.m16n8k16 (weights are the 16-row
+//     A operand, the batch is the 8-column B operand, fp32 accumulators) and issues the MMAs.
+// The decode per bit width is the cheapest exact one for the half-rate integer pipe and the shared-memory port:
+//   b = 4  per-row table of all 256 (centroid, centroid) pairs in shared memory, one copy per lane bank; the
+//          byte offset of a lookup is one PRMT of the packed word, one 32-bit LDS yields two weights.
+//   b = 2  the row's 4 centroids are the 8 source bytes of one PRMT; one PRMT yields two weights.
+//   b = 1  W^ = c0 + bit * (c1 - c0): the MMA multiplies by the signs (+1 / -1, one LOP3 per two weights, the
+//          shifts as multiplies on the FMA pipe) and the codebook is applied per output in the epilogue from
+//          D = sum(+-x) and S = sum(x).
+#include "kmq_common.cuh"
+#include "kmq_linear_variants.cuh"
+#include "kmq_mma_common.cuh"
+
+namespace kmq {
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kRows = kTileRows;
+constexpr int kPairEntryStride = 256;   // b = 4 tables: entry e, half h, lane l at e * 256 + h * 128 + l * 4
+constexpr int kTableBytes4 = 256 * kPairEntryStride;
+
+template <int BITS>
+struct TGeo {
+  static constexpr int kMmaPerWord = 8 / BITS;            // 16 k-slots per MMA = 4 lanes x 4 weights
+  static constexpr int kStepK = 512 / BITS;               // weights of one row per step
+  static constexpr int kWordK = 32 / BITS;
+  static constexpr int kChunkXBytes = 4 * kWordK * 2;     // activations under one 16-byte chunk of a row
+  static constexpr int kChunkStride = kChunkXBytes + 16;  // staged with 16 bytes of padding: no bank conflicts
+  static constexpr int kRowStride = 4 * kChunkStride;     // one batch row of one step
+  static constexpr int kPiecesPerRow = kStepK / 8;        // 16-byte pieces of x per batch row and step
+  static constexpr int kTableBytes = BITS == 4 ? kTableBytes4 : 0;
+  static constexpr int kStages = BITS == 4 ? 4 : 2;       // steps in flight per warp
+};
+
+template <int BITS, int MMAX>
+struct TSmem {
+  using G = TGeo<BITS>;
+  static constexpr int kXs = kWarps * MMAX * G::kRowStride;
+  static constexpr int kRed = kWarps * 32 * 16;
+  static constexpr int kRedS = kWarps * MMAX * 4;
+  static constexpr int kTotal = G::kTableBytes + kXs + kRed + kRedS;
+};
+
+// shared-memory byte offset (within one batch row of a warp's slice) of 16-byte piece `w` of a step
+template <int BITS>
+__device__ __forceinline__ int piece_offset(int w) {
+  using G = TGeo<BITS>;
+  constexpr int kPiecesPerChunk = G::kChunkXBytes / 16;
+  return (w / kPiecesPerChunk) * G::kChunkStride + (w % kPiecesPerChunk) * 16;
+}
+
+template <int BITS, int MMAX>
+__global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_t* __restrict__ packed,
+                                                                    const uint16_t* __restrict__ cb,
+                                                                    const uint16_t* __restrict__ x,
+                                                                    uint16_t* __restrict__ y, int64_t N, int64_t K,
+                                                                    int M) {
+  using G = TGeo<BITS>;
+  using SM = TSmem<BITS, MMAX>;
+  constexpr int Q = G::kMmaPerWord;
+  constexpr int STAGES = G::kStages;
+  // 16-byte pieces of x per lane and step, and whether they ride in the register ring with the weights
+  constexpr int kPieces = MMAX * G::kPiecesPerRow;
+  constexpr int NP = (kPieces + 31) / 32;
+  constexpr bool kPrefetchX = NP <= 2;
+
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  unsigned char* const tables = smem_raw;
+  unsigned char* const xs_warp = smem_raw + G::kTableBytes + (threadIdx.x >> 5) * (MMAX * G::kRowStride);
+  float* const red = reinterpret_cast<float*>(smem_raw + G::kTableBytes + SM::kXs);
+  float* const red_s = red + kWarps * 32 * 4;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int64_t row0 = (int64_t)blockIdx.x * kRows;
+  const int chunks = (int)(K / (4 * G::kWordK));   // 16-byte chunks per row
+  const int steps = (chunks + 3) >> 2;             // the layout pads every row to whole steps
+  // step s of this tile: 64 16-byte units, unit h * 32 + lane = row (g + 8h), chunk t
+  const uint4* __restrict__ tile = reinterpret_cast<const uint4*>(packed) + (int64_t)blockIdx.x * steps * 64 + lane;
+
+  // ---- x pieces of this lane: piece p = lane + 32 i -> batch row p / kPiecesPerRow, piece p % kPiecesPerRow
+  int px_k[NP], px_sm[NP];
+  const uint16_t* px_src[NP];
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    const int p = lane + 32 * i;
+    const int m = p / G::kPiecesPerRow, w = p % G::kPiecesPerRow;
+    px_k[i] = (p < kPieces && m < M) ? w * 8 : -1;   // k offset inside the step, or -1: nothing to copy
+    px_sm[i] = m * G::kRowStride + piece_offset<BITS>(w);
+    px_src[i] = x + (int64_t)m * K + w * 8;
+  }
+  auto load_x = [&](int s, uint4 (&v)[NP]) {
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      v[i] = make_uint4(0, 0, 0, 0);
+      if (px_k[i] >= 0 && (int64_t)s * G::kStepK + px_k[i] < K)
+        v[i] = __ldg(reinterpret_cast<const uint4*>(px_src[i] + (int64_t)s * G::kStepK));
+    }
+  };
+
+  // ---- ring: weights (and x pieces) of this warp's next kStages steps ----
+  constexpr int XS = kPrefetchX ? STAGES : 1;   // without prefetch one buffer, filled just before use
+  uint4 qa[STAGES], qb[STAGES], qx[XS][NP];
+#pragma unroll
+  for (int d = 0; d < STAGES; ++d) {
+    const int s = warp + d * kWarps;
+    qa[d] = qb[d] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) qx[kPrefetchX ? d : 0][i] = make_uint4(0, 0, 0, 0);
+    if (s < steps) {
+      qa[d] = ldg_stream_u4(tile + (int64_t)s * 64);
+      qb[d] = ldg_stream_u4(tile + (int64_t)s * 64 + 32);
+      if constexpr (kPrefetchX) load_x(s, qx[kPrefetchX ? d : 0]);
+    }
+  }
+
+  // ---- per-row decode state ----
+  Dec2 dg, dh;
+  if constexpr (BITS == 2) {
+    dg.init(cb + min(row0 + g, N - 1) * 4);
+    dh.init(cb + min(row0 + g + 8, N - 1) * 4);
+  }
+  if constexpr (BITS == 4) {
+    // entry e of row r: (C_r[e & 15], C_r[e >> 4]); the 4 lanes that share a row get one bank each
+    const int r8 = threadIdx.x & 7, half = (threadIdx.x >> 3) & 1;
+    const uint16_t* crow = cb + min(row0 + r8 + 8 * half, N - 1) * 16;
+    for (int e = threadIdx.x >> 4; e < 256; e += kThreads / 16) {
+      const uint32_t v = (uint32_t)__ldg(crow + (e & 15)) | ((uint32_t)__ldg(crow + (e >> 4)) << 16);
+      *reinterpret_cast<uint4*>(tables + e * kPairEntryStride + half * 128 + r8 * 16) = make_uint4(v, v, v, v);
+    }
+    __syncthreads();
+  }
+  const uint32_t lane4 = lane * 4;
+
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  float sacc[MMAX];
+#pragma unroll
+  for (int m = 0; m < MMAX; ++m) sacc[m] = 0.f;
+
+  // B fragments: lane (g, t) supplies batch row g; the columns of an MMA are independent, so lanes with
+  // g >= M re-read the last real row and their columns are never stored.
+  const unsigned char* const xb = xs_warp + min(g, M - 1) * G::kRowStride + t * G::kChunkStride;
+
+  for (int s0 = warp; s0 < steps; s0 += STAGES * kWarps) {
+#pragma unroll
+    for (int d = 0; d < STAGES; ++d) {
+      const int s = s0 + d * kWarps;
+      if (s < steps) {   // warp-uniform
+        // stage the activations under this step (zeros past K)
+        if constexpr (!kPrefetchX) load_x(s, qx[0]);
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < NP; ++i)
+          if (px_k[i] >= 0) *reinterpret_cast<uint4*>(xs_warp + px_sm[i]) = qx[kPrefetchX ? d : 0][i];
+        __syncwarp();
+
+        const uint32_t wa[4] = {qa[d].x, qa[d].y, qa[d].z, qa[d].w};
+        const uint32_t wb[4] = {qb[d].x, qb[d].y, qb[d].z, qb[d].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+          for (int q2 = 0; q2 < Q; q2 += 2) {
+            // 16 bytes of x = the 8 weights of two consecutive MMAs
+            const uint4 xv = *reinterpret_cast<const uint4*>(xb + (j * Q + q2) * 8);
+#pragma unroll
+            for (int qq = 0; qq < 2; ++qq) {
+              const int q = q2 + qq;
+              uint32_t a0, a1, a2, a3;
+              if constexpr (BITS == 2) {
+                dg.pair(wa[j], q, a0, a2);
+                dh.pair(wb[j], q, a1, a3);
+              } else if constexpr (BITS == 4) {
+                // index byte k of the word -> byte offset (byte << 8) | lane * 4: result bytes (lane4, byte k, 0, 0)
+                const uint32_t s0b = 0x5504u | ((2 * q) << 4), s1b = 0x5504u | ((2 * q + 1) << 4);
+                a0 = *reinterpret_cast<const uint32_t*>(tables + prmt(wa[j], lane4, s0b));
+                a2 = *reinterpret_cast<const uint32_t*>(tables + prmt(wa[j], lane4, s1b));
+                a1 = *reinterpret_cast<const uint32_t*>(tables + 128 + prmt(wb[j], lane4, s0b));
+                a3 = *reinterpret_cast<const uint32_t*>(tables + 128 + prmt(wb[j], lane4, s1b));
+              } else {
+                // shift by c puts weights (2c, 2c+1) of the word on the two sign bits; c = 2q and 2q + 1
+                const uint32_t m0 = kPow2[2 * q], m1 = kPow2[2 * q + 1];
+                a0 = and_or(wa[j] * m0, 0x80008000u, 0x3F803F80u);
+                a2 = and_or(wa[j] * m1, 0x80008000u, 0x3F803F80u);
+                a1 = and_or(wb[j] * m0, 0x80008000u, 0x3F803F80u);
+                a3 = and_or(wb[j] * m1, 0x80008000u, 0x3F803F80u);
+              }
+              mma_bf16_16816(acc, a0, a1, a2, a3, qq ? xv.z : xv.x, qq ? xv.w : xv.y);
+            }
+          }
+        }
+        if constexpr (BITS == 1) {
+          // S[m] = sum_k x[m,k]: the 512 staged activations of a batch row as two 16x16 A tiles times a matrix
+          // of ones give 16 row sums each; the order of the addends is irrelevant.
+#pragma unroll
+          for (int m = 0; m < MMAX; ++m) {
+            if (m < M) {
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                const uint4 v =
+                    *reinterpret_cast<const uint4*>(xs_warp + m * G::kRowStride + piece_offset<BITS>(lane + 32 * h));
+                float tmp[4] = {0.f, 0.f, 0.f, 0.f};
+                mma_bf16_16816(tmp, v.x, v.y, v.z, v.w, 0x3F803F80u, 0x3F803F80u);
+                sacc[m] += tmp[0] + tmp[2];   // rows g and g + 8 (identical in every column)
+              }
+            }
+          }
+        }
+        // refill this stage for the step kStages rounds ahead
+        const int s2 = s + STAGES * kWarps;
+        if (s2 < steps) {
+          qa[d] = ldg_stream_u4(tile + (int64_t)s2 * 64);
+          qb[d] = ldg_stream_u4(tile + (int64_t)s2 * 64 + 32);
+          if constexpr (kPrefetchX) load_x(s2, qx[kPrefetchX ? d : 0]);
+        }
+      }
+    }
+  }
+
+  // ---- add the partial sums of the warps, apply the codebook (b = 1), store ----
+  *reinterpret_cast<float4*>(red + (warp * 32 + lane) * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+  if constexpr (BITS == 1) {
+#pragma unroll
+    for (int m = 0; m < MMAX; ++m) {
+      float v = sacc[m];
+      v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
+      v += __shfl_xor_sync(0xFFFFFFFFu, v, 8);
+      v += __shfl_xor_sync(0xFFFFFFFFu, v, 16);
+      if (lane == 0) red_s[warp * MMAX + m] = v;   // lanes with t = 0 cover every row once
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < kRows * 8) {
+    const int r = threadIdx.x & 15, m = threadIdx.x >> 4;   // consecutive threads -> consecutive output rows
+    const int64_t n = row0 + r;
+    if (m < M && n < N) {
+      const int src_lane = (r & 7) * 4 + (m >> 1), src_reg = (r >> 3) * 2 + (m & 1);
+      float v = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) v += red[(w * 32 + src_lane) * 4 + src_reg];
+      if constexpr (BITS == 1) {
+        float sx = 0.f;
+        const int mm = m < MMAX ? m : 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) sx += red_s[w * MMAX + mm];
+        // v = T0 - T1, sx = T0 + T1 with T_i the sum of the activations whose weight has index i
+        const uint32_t c = __ldg(reinterpret_cast<const uint32_t*>(cb + n * 2));
+        const float c0 = bf16_bits_to_float(c & 0xFFFFu), c1 = bf16_bits_to_float(c >> 16);
+        v = fmaf(c0, 0.5f * (sx + v), c1 * (0.5f * (sx - v)));
+      }
+      y[(int64_t)m * N + n] = (uint16_t)float_to_bf16_bits(v);
+    }
+  }
+}
+
+template <int BITS, int MMAX>
+cudaError_t launch_one(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                       int64_t K, int M, cudaStream_t s) {
+  constexpr int smem = TSmem<BITS, MMAX>::kTotal;
+  static bool configured[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    cudaError_t e =
+        cudaFuncSetAttribute(linear_tiled_kernel<BITS, MMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  const unsigned grid = (unsigned)((N + kRows - 1) / kRows);
+  linear_tiled_kernel<BITS, MMAX><<<grid, kThreads, smem, s>>>(packed, cb, x, y, N, K, M);
+  return cudaGetLastError();
+}
+
+template <int BITS>
+cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                        int64_t K, int M, cudaStream_t s) {
+  if (M == 1) return launch_one<BITS, 1>(packed, cb, x, y, N, K, M, s);
+  if (M == 2) return launch_one<BITS, 2>(packed, cb, x, y, N, K, M, s);
+  if (M <= 4) return launch_one<BITS, 4>(packed, cb, x, y, N, K, M, s);
+  return launch_one<BITS, 8>(packed, cb, x, y, N, K, M, s);
+}
+
+}  // namespace
+
+// Tuned layout.  Batches larger than 8 are processed 8 rows at a time (one launch each).
+cudaError_t launch_linear_tiled(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                                int64_t K, int bits, int64_t M, cudaStream_t s) {
+  for (int64_t m0 = 0; m0 < M; m0 += 8) {
+    const int mc = (int)(M - m0 < 8 ? M - m0 : 8);
+    const uint16_t* xp = x + m0 * K;
+    uint16_t* yp = y + m0 * N;
+    cudaError_t e;
+    if (bits == 1) e = launch_bits<1>(packed, cb, xp, yp, N, K, mc, s);
+    else if (bits == 2) e = launch_bits<2>(packed, cb, xp, yp, N, K, mc, s);
+    else e = launch_bits<4>(packed, cb, xp, yp, N, K, mc, s);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace kmq

@@ -18,6 +18,7 @@ KMQ_OK = 0
 KMQ_ERR_NULL, KMQ_ERR_BITS, KMQ_ERR_SHAPE, KMQ_ERR_ALIGN = 1, 2, 3, 4
 KMQ_ERR_WORKSPACE, KMQ_ERR_LAYOUT, KMQ_ERR_CUDA = 5, 6, 7
 KMQ_LAYOUT_CANONICAL = 0
+KMQ_LAYOUT_TUNED = 1
 
 _i64, _int, _ptr, _sz = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t
 
@@ -26,9 +27,9 @@ SIGNATURES = {
     "kmq_version": (_int, []),
     "kmq_status_string": (ctypes.c_char_p, [_int]),
     "kmq_packed_bytes": (_sz, [_i64, _i64, _int, _int]),
-    "kmq_workspace_bytes": (_sz, [_i64, _i64, _int, _i64]),
-    "kmq_linear_num_launches": (_int, [_i64, _i64, _int, _i64]),
-    "kmq_linear_variant": (ctypes.c_char_p, [_i64, _i64, _int, _i64]),
+    "kmq_workspace_bytes": (_sz, [_i64, _i64, _int, _i64, _int]),
+    "kmq_linear_num_launches": (_int, [_i64, _i64, _int, _i64, _int]),
+    "kmq_linear_variant": (ctypes.c_char_p, [_i64, _i64, _int, _i64, _int]),
     "kmq_pack": (_int, [_ptr, _i64, _i64, _int, _int, _ptr, _ptr]),
     "kmq_unpack": (_int, [_ptr, _i64, _i64, _int, _int, _ptr, _ptr]),
     "kmq_linear": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr, _sz, _ptr]),
@@ -93,16 +94,16 @@ def kmq_packed_bytes(N, K, bits, layout=KMQ_LAYOUT_CANONICAL) -> int:
     return lib().kmq_packed_bytes(N, K, bits, layout)
 
 
-def kmq_workspace_bytes(N, K, bits, M) -> int:
-    return lib().kmq_workspace_bytes(N, K, bits, M)
+def kmq_workspace_bytes(N, K, bits, M, layout=KMQ_LAYOUT_CANONICAL) -> int:
+    return lib().kmq_workspace_bytes(N, K, bits, M, layout)
 
 
-def kmq_linear_num_launches(N, K, bits, M) -> int:
-    return lib().kmq_linear_num_launches(N, K, bits, M)
+def kmq_linear_num_launches(N, K, bits, M, layout=KMQ_LAYOUT_CANONICAL) -> int:
+    return lib().kmq_linear_num_launches(N, K, bits, M, layout)
 
 
-def kmq_linear_variant(N, K, bits, M) -> str:
-    return lib().kmq_linear_variant(N, K, bits, M).decode()
+def kmq_linear_variant(N, K, bits, M, layout=KMQ_LAYOUT_CANONICAL) -> str:
+    return lib().kmq_linear_variant(N, K, bits, M, layout).decode()
 
 
 def kmq_pack(idx, N, K, bits, packed, layout=KMQ_LAYOUT_CANONICAL, stream=None, check=True) -> int:

@@ -26,37 +26,53 @@ def to_dev_u16(a: np.ndarray) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda()
 
 
-def gpu_pack(idx: np.ndarray, bits: int) -> torch.Tensor:
+def gpu_pack(idx: np.ndarray, bits: int, layout: int = kmq.KMQ_LAYOUT_CANONICAL) -> torch.Tensor:
+    """Pack on the GPU into a buffer with canary bands; returns the payload view."""
     N, K = idx.shape
     d_idx = torch.from_numpy(np.ascontiguousarray(idx)).cuda()
-    packed = torch.empty(kmq.kmq_packed_bytes(N, K, bits) // 4, dtype=torch.int32, device="cuda")
-    kmq.kmq_pack(d_idx, N, K, bits, packed)
-    return packed
+    nbytes = kmq.kmq_packed_bytes(N, K, bits, layout)
+    buf, off = dev_bytes(nbytes)
+    assert (buf.data_ptr() + off) % 16 == 0
+    kmq.kmq_pack(d_idx, N, K, bits, buf.data_ptr() + off, layout=layout)
+    torch.cuda.synchronize()
+    assert canaries_intact(buf, off, nbytes), "pack wrote outside its buffer"
+    return buf[off:off + nbytes].view(torch.int32)
+
+
+def gpu_unpack(packed: torch.Tensor, N: int, K: int, bits: int, layout: int = kmq.KMQ_LAYOUT_CANONICAL) -> np.ndarray:
+    nbytes = N * K
+    buf, off = dev_bytes(nbytes)
+    kmq.kmq_unpack(packed, N, K, bits, buf.data_ptr() + off, layout=layout)
+    torch.cuda.synchronize()
+    assert canaries_intact(buf, off, nbytes), "unpack wrote outside idx"
+    return buf[off:off + nbytes].cpu().numpy().reshape(N, K)
 
 
 def packed_to_numpy(packed: torch.Tensor, N: int) -> np.ndarray:
     return packed.cpu().numpy().view(np.uint32).reshape(N, -1)
 
 
-def gpu_dequant(packed: torch.Tensor, cb: np.ndarray, N: int, K: int, bits: int) -> np.ndarray:
+def gpu_dequant(packed: torch.Tensor, cb: np.ndarray, N: int, K: int, bits: int,
+                layout: int = kmq.KMQ_LAYOUT_CANONICAL) -> np.ndarray:
     d_cb = to_dev_u16(cb)
     nbytes = N * K * 2
     buf, off = dev_bytes(nbytes)
-    kmq.kmq_dequant_to_bf16(packed, d_cb, buf.data_ptr() + off, N, K, bits)
+    kmq.kmq_dequant_to_bf16(packed, d_cb, buf.data_ptr() + off, N, K, bits, layout=layout)
     torch.cuda.synchronize()
     assert canaries_intact(buf, off, nbytes), "dequant wrote outside W"
     return buf[off:off + nbytes].cpu().numpy().view(np.uint16).reshape(N, K)
 
 
-def gpu_linear(packed: torch.Tensor, cb: np.ndarray, x: np.ndarray, N: int, K: int, bits: int) -> np.ndarray:
+def gpu_linear(packed: torch.Tensor, cb: np.ndarray, x: np.ndarray, N: int, K: int, bits: int,
+               layout: int = kmq.KMQ_LAYOUT_CANONICAL) -> np.ndarray:
     M = x.shape[0]
     d_cb, d_x = to_dev_u16(cb), to_dev_u16(x)
     nbytes = M * N * 2
     buf, off = dev_bytes(nbytes)
-    ws_bytes = kmq.kmq_workspace_bytes(N, K, bits, M)
+    ws_bytes = kmq.kmq_workspace_bytes(N, K, bits, M, layout)
     wsbuf, wsoff = dev_bytes(max(ws_bytes, 16))
     kmq.kmq_linear(packed, d_cb, d_x, buf.data_ptr() + off, N, K, bits, M,
-                   wsbuf.data_ptr() + wsoff, ws_bytes)
+                   wsbuf.data_ptr() + wsoff, ws_bytes, layout=layout)
     torch.cuda.synchronize()
     assert canaries_intact(buf, off, nbytes), "linear wrote outside y"
     assert canaries_intact(wsbuf, wsoff, max(ws_bytes, 16)), "linear wrote outside its workspace"

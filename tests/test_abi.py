@@ -49,6 +49,13 @@ def test_sizes_and_strings():
     assert kmq.kmq_linear_num_launches(4096, 4095, 4, 1) == 0
     assert isinstance(kmq.kmq_linear_variant(4096, 4096, 2, 1), str)
     assert kmq.kmq_workspace_bytes(4096, 4096, 3, 1) == 0
+    T = kmq.KMQ_LAYOUT_TUNED
+    assert kmq.kmq_packed_bytes(4096, 4096, 2, layout=T) == 4096 * 4096 // 4      # whole tiles and steps: no padding
+    assert kmq.kmq_packed_bytes(17, 32, 1, layout=T) == 2 * 1 * 1024               # 2 tiles x 1 step x 1 KB
+    assert kmq.kmq_packed_bytes(16, 8 * 17, 4, layout=T) == 1 * 2 * 1024            # 17 words per row -> 2 steps
+    assert kmq.kmq_linear_num_launches(4096, 4096, 2, 17, layout=T) == 3
+    assert kmq.kmq_linear_variant(4096, 4096, 2, 1, layout=7) == "invalid"
+    assert kmq.kmq_linear_variant(4096, 4096, 2, 1, layout=T) != kmq.kmq_linear_variant(4096, 4096, 2, 1)
 
 
 A = 0x1000  # a non-NULL, 16-byte aligned fake address; never dereferenced: validation fails first

@@ -22,18 +22,34 @@ def random_layer(rng, N, K, bits, M):
     return idx, cb, x
 
 
+LAYOUTS = (kmq.KMQ_LAYOUT_CANONICAL, kmq.KMQ_LAYOUT_TUNED)
+
+
 def check_all(idx, cb, x, bits, what=""):
+    """Both packed layouts.  The canonical words must equal the oracle's bit for bit; the tuned words are defined
+    only through what they decode to (indices, weights), which must be exact, and their padding must be zero."""
     N, K = idx.shape
     ref_packed = orc.pack_canonical(idx, bits)
-    packed = gu.gpu_pack(idx, bits)
-    assert np.array_equal(gu.packed_to_numpy(packed, N), ref_packed), f"{what}: packed words differ"
-    w = gu.gpu_dequant(packed, cb, N, K, bits)
-    assert np.array_equal(w, orc.dequant_bits(ref_packed, cb, K, bits)), f"{what}: dequantised weights differ"
-    y = gu.gpu_linear(packed, cb, x, N, K, bits)
+    ref_w = orc.dequant_bits(ref_packed, cb, K, bits)
     y_ref, s = orc.linear_f64(ref_packed, cb, x, K, bits)
-    ratio = orc.check_linear(y, y_ref, s)
-    assert ratio <= 1.0, f"{what}: error/tolerance = {ratio}"
-    return ratio
+    worst = 0.0
+    for layout in LAYOUTS:
+        tag = f"{what} layout={layout}"
+        packed = gu.gpu_pack(idx, bits, layout)
+        if layout == kmq.KMQ_LAYOUT_CANONICAL:
+            assert np.array_equal(gu.packed_to_numpy(packed, N), ref_packed), f"{tag}: packed words differ"
+        else:
+            assert np.array_equal(gu.gpu_unpack(packed, N, K, bits, layout), idx), f"{tag}: unpack(pack(idx)) != idx"
+            pop = int(np.unpackbits(packed.cpu().numpy().view(np.uint8)).sum())
+            assert pop == int(np.unpackbits(ref_packed.view(np.uint8)).sum()), f"{tag}: padding is not zero"
+        w = gu.gpu_dequant(packed, cb, N, K, bits, layout)
+        assert np.array_equal(w, ref_w), f"{tag}: dequantised weights differ"
+        y = gu.gpu_linear(packed, cb, x, N, K, bits, layout)
+        ratio = orc.check_linear(y, y_ref, s)
+        assert ratio <= 1.0, (f"{tag}: error/tolerance = {ratio} "
+                              f"[{kmq.kmq_linear_variant(N, K, bits, x.shape[0], layout)}]")
+        worst = max(worst, ratio)
+    return worst
 
 
 # ---- configuration 1 (tiny correctness layer), all bit widths ----
