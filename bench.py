@@ -142,9 +142,10 @@ class Case:
         self.layer = layer
         dev = torch.device("cuda")
         idx = torch.from_numpy(layer["idx"]).to(dev)
-        words = kmq.kmq_packed_bytes(N, K, bits) // 4
+        self.layout = kmq.KMQ_LAYOUT_TUNED                         # the layout the fast kernels read
+        words = kmq.kmq_packed_bytes(N, K, bits, self.layout) // 4
         self.packed = torch.empty((self.pool, words), dtype=torch.int32, device=dev)
-        kmq.kmq_pack(idx, N, K, bits, self.packed[0])              # a1: offline packing, on the GPU
+        kmq.kmq_pack(idx, N, K, bits, self.packed[0], layout=self.layout)   # a1: offline packing, on the GPU
         self.packed[1:] = self.packed[0]
         del idx
         cb = torch.from_numpy(layer["codebooks"].view(np.int16)).to(dev)
@@ -155,19 +156,20 @@ class Case:
         self.x = self.x_host.to(dev)
         self.y = torch.zeros((self.pool, M, N), dtype=torch.int16, device=dev)
         self.y_host = torch.zeros((self.pool, M, N), dtype=torch.int16).pin_memory()
-        self.ws_bytes = kmq.kmq_workspace_bytes(N, K, bits, M)
+        self.ws_bytes = kmq.kmq_workspace_bytes(N, K, bits, M, self.layout)
         self.ws = torch.empty(max(self.ws_bytes, 16), dtype=torch.uint8, device=dev)
-        self.launches = kmq.kmq_linear_num_launches(N, K, bits, M)
-        self.variant = kmq.kmq_linear_variant(N, K, bits, M)
+        self.launches = kmq.kmq_linear_num_launches(N, K, bits, M, self.layout)
+        self.variant = kmq.kmq_linear_variant(N, K, bits, M, self.layout)
         self.kmq = kmq
 
     def call(self, i):
         self.kmq.kmq_linear(self.packed[i], self.cb[i], self.x[i], self.y[i], self.N, self.K, self.bits, self.M,
-                            self.ws, self.ws_bytes)
+                            self.ws, self.ws_bytes, layout=self.layout)
 
     def call_host(self, i):
         self.kmq.kmq_linear_host(self.packed[i], self.cb[i], self.x_host[i].data_ptr(), self.y_host[i].data_ptr(),
-                                 self.N, self.K, self.bits, self.M, self.x[i], self.y[i], self.ws, self.ws_bytes)
+                                 self.N, self.K, self.bits, self.M, self.x[i], self.y[i], self.ws, self.ws_bytes,
+                                 layout=self.layout)
 
 
 def run_library(args):
@@ -256,6 +258,15 @@ def run_library(args):
 
     # ---- end to end through the host-buffer entry point (H2D of x, D2H of y inside) ----
     e2e_steps = max(1, min(args.steps, 5))
+    if args.quick:
+        sampler.stop_flag = True
+        if rank == 0:
+            for c, ms in zip(cases, per_case_ms):
+                print(f"{c.name} b={c.bits} M={c.M} [{c.variant}]: {ms * 1e3 / c.pool:.3f} us/call, "
+                      f"{c.bytes / (ms * 1e-3 / c.pool) / 1e9:.1f} GB/s")
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     with torch.cuda.stream(stream):
         for c in cases:
             c.call_host(0)
@@ -324,7 +335,8 @@ def run_library(args):
         "config": {"workload": f"{args.workload}: {WORKLOAD_TEXT[args.workload]}",
                    "calls_per_step": step_calls, "bytes_per_step": step_bytes,
                    "l2": "inputs larger than L2: every call of a step uses its own weight set, pool >= 2 x 126 MB",
-                   "launch": "CUDA graph per case, replayed once per step", "multi_gpu": "replicas only"},
+                   "launch": "CUDA graph per case, replayed once per step", "multi_gpu": "replicas only",
+                   "packed_layout": "tuned (tile-major), packed once by kmq_pack before the timed region"},
         "frac_of_measured_hbm": round(value / world / peak_gbs, 4),
         "us_per_call_mean": round(elapsed_ms * 1e3 / args.steps / step_calls, 3),
         "per_case": per_case,
@@ -432,6 +444,8 @@ def main():
     ap.add_argument("--impl", default="kmq", choices=["kmq", "reference"])
     ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS))
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--quick", action="store_true",
+                    help="kernel timing only (no end-to-end leg, CPU baseline or parity check): for profiler runs")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
