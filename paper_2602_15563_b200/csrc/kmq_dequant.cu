@@ -9,63 +9,84 @@ namespace {
 
 // The 8*BITS bits that hold weights 8c .. 8c+7 of row n, fields LSB first.
 template <int BITS, bool TUNED>
-__device__ __forceinline__ uint32_t load_chunk_bits(const uint32_t* __restrict__ packed, int64_t n, int64_t wpr,
-                                                    int64_t steps, int64_t c) {
+__device__ __forceinline__ uint32_t load_chunk_bits(const uint32_t* __restrict__ row_words, int c) {
+  // row_words: canonical -> first word of the row; tuned -> word 0 of the row inside its tile (see word_at)
+  constexpr int CPW = 4 / BITS;   // 8-weight chunks per word (b = 4: 1, b = 2: 2, b = 1: 4)
   if constexpr (TUNED) {
-    // the fields of a chunk are spread over its word: permute the word back, then cut the chunk out
-    constexpr int CPW = 4 / BITS;   // 8-weight chunks per word
-    const uint32_t w = canonical_from_tuned<BITS>(__ldg(packed + tuned_word_index(n, c / CPW, steps)));
-    if constexpr (BITS == 4) return w;
-    return (w >> ((int)(c % CPW) * 8 * BITS)) & ((1u << (8 * BITS)) - 1u);
+    const int j = c / CPW, q = c % CPW;
+    // word j of the row: step j / 16 is 256 words further, then the word inside the row's 64 bytes
+    const uint32_t t = __ldg(row_words + (int64_t)(j >> 4) * 256 + (j & 15));
+    if constexpr (BITS == 4) {
+      return t;
+    } else {
+      constexpr uint32_t MASK = (1u << BITS) - 1u;
+      uint32_t v = 0;
+#pragma unroll
+      for (int qq = 0; qq < CPW; ++qq) {   // q selects one of CPW compile-time extraction patterns
+        if (qq == q) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) v |= ((t >> field_pos<BITS>(8 * qq + i, true)) & MASK) << (i * BITS);
+        }
+      }
+      return v;
+    }
   } else if constexpr (BITS == 4) {
-    return __ldg(packed + n * wpr + c);
+    return __ldg(row_words + c);
   } else if constexpr (BITS == 2) {
-    return __ldg(reinterpret_cast<const uint16_t*>(packed + n * wpr) + c);
+    return __ldg(reinterpret_cast<const uint16_t*>(row_words) + c);
   } else {
-    return __ldg(reinterpret_cast<const uint8_t*>(packed + n * wpr) + c);
+    return __ldg(reinterpret_cast<const uint8_t*>(row_words) + c);
   }
 }
 
+// One CTA walks rows (grid-stride); inside a row every thread turns 8 weights into one 16-byte streaming store,
+// consecutive threads writing consecutive pieces.
 template <int BITS, bool TUNED>
 __global__ void __launch_bounds__(256) dequant_kernel(const uint32_t* __restrict__ packed,
                                                       const uint16_t* __restrict__ cb, uint16_t* __restrict__ W,
                                                       int64_t N, int64_t K) {
   constexpr int Q = 1 << BITS;
-  const int64_t cpr = K >> 3;            // 8-weight chunks per row
-  const int64_t wpr = K / (32 / BITS);   // words per row
+  const int cpr = (int)(K >> 3);                 // 8-weight chunks per row
+  const int64_t wpr = K / (32 / BITS);           // words per row
   const int64_t steps = tuned_steps(wpr);
-  const int64_t total = N * cpr;
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t chunk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; chunk < total; chunk += stride) {
-    const int64_t n = chunk / cpr;
-    const int64_t c = chunk - n * cpr;
-    const uint32_t v = load_chunk_bits<BITS, TUNED>(packed, n, wpr, steps, c);
-    uint32_t o[4];
-    if constexpr (BITS == 1) {
-      // codebook = 4 bytes {c0, c1}; a selector nibble pair picks bytes (2i, 2i+1)
-      const uint32_t cw = __ldg(reinterpret_cast<const uint32_t*>(cb + n * Q));
-#pragma unroll
-      for (int p = 0; p < 4; ++p) {
-        const uint32_t i0 = (v >> (2 * p)) & 1u, i1 = (v >> (2 * p + 1)) & 1u;
-        o[p] = __byte_perm(cw, cw, 0x1010u + i0 * 0x22u + i1 * 0x2200u);
-      }
-    } else if constexpr (BITS == 2) {
-      // codebook = 8 bytes {c0,c1 | c2,c3}: byte pair (2i, 2i+1) of the two words
-      const uint2 cw = __ldg(reinterpret_cast<const uint2*>(cb + n * Q));
-#pragma unroll
-      for (int p = 0; p < 4; ++p) {
-        const uint32_t i0 = (v >> (4 * p)) & 3u, i1 = (v >> (4 * p + 2)) & 3u;
-        o[p] = __byte_perm(cw.x, cw.y, 0x1010u + i0 * 0x22u + i1 * 0x2200u);
-      }
-    } else {
-      const uint16_t* row_cb = cb + n * Q;
-#pragma unroll
-      for (int p = 0; p < 4; ++p) {
-        const uint32_t i0 = (v >> (8 * p)) & 15u, i1 = (v >> (8 * p + 4)) & 15u;
-        o[p] = (uint32_t)__ldg(row_cb + i0) | ((uint32_t)__ldg(row_cb + i1) << 16);
-      }
+  for (int64_t n = blockIdx.x; n < N; n += gridDim.x) {
+    const uint32_t* row_words =
+        TUNED ? packed + ((n >> 4) * steps * kTileRows + (n & 15)) * 16 : packed + n * wpr;
+    const uint16_t* row_cb = cb + n * Q;
+    uint32_t c0 = 0, c1 = 0;
+    if constexpr (BITS == 1) c0 = __ldg(reinterpret_cast<const uint32_t*>(row_cb));
+    if constexpr (BITS == 2) {
+      const uint2 cw = __ldg(reinterpret_cast<const uint2*>(row_cb));
+      c0 = cw.x;
+      c1 = cw.y;
     }
-    stg_stream_u4(reinterpret_cast<uint4*>(W + n * K + c * 8), make_uint4(o[0], o[1], o[2], o[3]));
+    uint4* out = reinterpret_cast<uint4*>(W + n * K);
+    for (int c = threadIdx.x; c < cpr; c += 256) {
+      const uint32_t v = load_chunk_bits<BITS, TUNED>(row_words, c);
+      uint32_t o[4];
+      if constexpr (BITS == 1) {
+        // codebook = 4 bytes {c0, c1}; a selector nibble pair picks bytes (2i, 2i+1)
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+          const uint32_t i0 = (v >> (2 * p)) & 1u, i1 = (v >> (2 * p + 1)) & 1u;
+          o[p] = __byte_perm(c0, c0, 0x1010u + i0 * 0x22u + i1 * 0x2200u);
+        }
+      } else if constexpr (BITS == 2) {
+        // codebook = 8 bytes {c0,c1 | c2,c3}: byte pair (2i, 2i+1) of the two words
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+          const uint32_t i0 = (v >> (4 * p)) & 3u, i1 = (v >> (4 * p + 2)) & 3u;
+          o[p] = __byte_perm(c0, c1, 0x1010u + i0 * 0x22u + i1 * 0x2200u);
+        }
+      } else {
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+          const uint32_t i0 = (v >> (8 * p)) & 15u, i1 = (v >> (8 * p + 4)) & 15u;
+          o[p] = (uint32_t)__ldg(row_cb + i0) | ((uint32_t)__ldg(row_cb + i1) << 16);
+        }
+      }
+      stg_stream_u4(out + c, make_uint4(o[0], o[1], o[2], o[3]));
+    }
   }
 }
 
@@ -75,11 +96,9 @@ cudaError_t launch_dequant(const uint32_t* packed, const uint16_t* cb, uint16_t*
                            int layout, cudaStream_t s) {
   const DeviceInfo* di = device_info();
   if (!di) return cudaGetLastError();
-  const int64_t total = N * (K >> 3);
-  int64_t blocks = (total + 255) / 256;
-  const int64_t cap = (int64_t)di->sm_count * 32;
+  int64_t blocks = N;
+  const int64_t cap = (int64_t)di->sm_count * 8;   // 8 resident CTAs of 256 threads per SM
   if (blocks > cap) blocks = cap;
-  if (blocks < 1) blocks = 1;
   const bool tuned = layout == KMQ_LAYOUT_TUNED;
   if (bits == 1 && tuned) dequant_kernel<1, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
   else if (bits == 1) dequant_kernel<1, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
