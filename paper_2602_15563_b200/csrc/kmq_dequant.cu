@@ -7,45 +7,54 @@
 namespace kmq {
 namespace {
 
-// The 8*BITS bits that hold weights 8c .. 8c+7 of row n, fields LSB first.
-template <int BITS, bool TUNED>
-__device__ __forceinline__ uint32_t load_chunk_bits(const uint32_t* __restrict__ row_words, int c) {
-  // row_words: canonical -> first word of the row; tuned -> word 0 of the row inside its tile (see word_at)
-  constexpr int CPW = 4 / BITS;   // 8-weight chunks per word (b = 4: 1, b = 2: 2, b = 1: 4)
-  if constexpr (TUNED) {
-    const int j = c / CPW, q = c % CPW;
-    // word j of the row: step j / 16 is 256 words further, then the word inside the row's 64 bytes
-    const uint32_t t = __ldg(row_words + (int64_t)(j >> 4) * 256 + (j & 15));
-    if constexpr (BITS == 4) {
-      return t;
-    } else {
-      constexpr uint32_t MASK = (1u << BITS) - 1u;
-      uint32_t v = 0;
+// 8 weights (8*BITS index bits, fields LSB first) -> 8 bf16 = one 16-byte value.
+template <int BITS>
+__device__ __forceinline__ uint4 decode8(uint32_t v, uint32_t c0, uint32_t c1, const uint16_t* __restrict__ row_cb) {
+  uint32_t o[4];
+  if constexpr (BITS == 1) {
+    // codebook = 4 bytes {c0, c1}; a selector nibble pair picks bytes (2i, 2i+1)
 #pragma unroll
-      for (int qq = 0; qq < CPW; ++qq) {   // q selects one of CPW compile-time extraction patterns
-        if (qq == q) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) v |= ((t >> field_pos<BITS>(8 * qq + i, true)) & MASK) << (i * BITS);
-        }
-      }
-      return v;
+    for (int p = 0; p < 4; ++p) {
+      const uint32_t i0 = (v >> (2 * p)) & 1u, i1 = (v >> (2 * p + 1)) & 1u;
+      o[p] = __byte_perm(c0, c0, 0x1010u + i0 * 0x22u + i1 * 0x2200u);
     }
-  } else if constexpr (BITS == 4) {
-    return __ldg(row_words + c);
   } else if constexpr (BITS == 2) {
-    return __ldg(reinterpret_cast<const uint16_t*>(row_words) + c);
+    // codebook = 8 bytes {c0,c1 | c2,c3}: byte pair (2i, 2i+1) of the two words
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      const uint32_t i0 = (v >> (4 * p)) & 3u, i1 = (v >> (4 * p + 2)) & 3u;
+      o[p] = __byte_perm(c0, c1, 0x1010u + i0 * 0x22u + i1 * 0x2200u);
+    }
   } else {
-    return __ldg(reinterpret_cast<const uint8_t*>(row_words) + c);
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      const uint32_t i0 = (v >> (8 * p)) & 15u, i1 = (v >> (8 * p + 4)) & 15u;
+      o[p] = (uint32_t)__ldg(row_cb + i0) | ((uint32_t)__ldg(row_cb + i1) << 16);
+    }
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+template <int BITS>
+__device__ __forceinline__ void load_codebook(const uint16_t* __restrict__ row_cb, uint32_t& c0, uint32_t& c1) {
+  c0 = c1 = 0;
+  if constexpr (BITS == 1) c0 = __ldg(reinterpret_cast<const uint32_t*>(row_cb));
+  if constexpr (BITS == 2) {
+    const uint2 cw = __ldg(reinterpret_cast<const uint2*>(row_cb));
+    c0 = cw.x;
+    c1 = cw.y;
   }
 }
 
 // One CTA walks rows (grid-stride); inside a row every thread turns 8 weights into one 16-byte streaming store,
-// consecutive threads writing consecutive pieces.
+// consecutive threads writing consecutive pieces.  In the tuned layout the row's words come in 64-byte runs, one
+// per 1 KB step of its tile, and the 8 fields of a chunk are cut out of the word after one shift.
 template <int BITS, bool TUNED>
-__global__ void __launch_bounds__(256) dequant_kernel(const uint32_t* __restrict__ packed,
-                                                      const uint16_t* __restrict__ cb, uint16_t* __restrict__ W,
-                                                      int64_t N, int64_t K) {
+__global__ void __launch_bounds__(256) dequant_rows_kernel(const uint32_t* __restrict__ packed,
+                                                           const uint16_t* __restrict__ cb, uint16_t* __restrict__ W,
+                                                           int64_t N, int64_t K) {
   constexpr int Q = 1 << BITS;
+  constexpr int CPW = 4 / BITS;                  // 8-weight chunks per word
   const int cpr = (int)(K >> 3);                 // 8-weight chunks per row
   const int64_t wpr = K / (32 / BITS);           // words per row
   const int64_t steps = tuned_steps(wpr);
@@ -53,39 +62,37 @@ __global__ void __launch_bounds__(256) dequant_kernel(const uint32_t* __restrict
     const uint32_t* row_words =
         TUNED ? packed + ((n >> 4) * steps * kTileRows + (n & 15)) * 16 : packed + n * wpr;
     const uint16_t* row_cb = cb + n * Q;
-    uint32_t c0 = 0, c1 = 0;
-    if constexpr (BITS == 1) c0 = __ldg(reinterpret_cast<const uint32_t*>(row_cb));
-    if constexpr (BITS == 2) {
-      const uint2 cw = __ldg(reinterpret_cast<const uint2*>(row_cb));
-      c0 = cw.x;
-      c1 = cw.y;
-    }
+    uint32_t c0, c1;
+    load_codebook<BITS>(row_cb, c0, c1);
     uint4* out = reinterpret_cast<uint4*>(W + n * K);
     for (int c = threadIdx.x; c < cpr; c += 256) {
-      const uint32_t v = load_chunk_bits<BITS, TUNED>(row_words, c);
-      uint32_t o[4];
-      if constexpr (BITS == 1) {
-        // codebook = 4 bytes {c0, c1}; a selector nibble pair picks bytes (2i, 2i+1)
+      uint32_t v;
+      if constexpr (TUNED) {
+        const int j = c / CPW, q = c % CPW;
+        const uint32_t t = __ldg(row_words + (int64_t)(j >> 4) * 256 + (j & 15));
+        if constexpr (BITS == 4) {
+          v = t;
+        } else if constexpr (BITS == 2) {
+          // field 4p + c' at bits 2p + 8c'; chunk q holds p = 2q, 2q+1: shift them down to p = 0, 1
+          const uint32_t u = t >> (4 * q);
+          v = 0;
 #pragma unroll
-        for (int p = 0; p < 4; ++p) {
-          const uint32_t i0 = (v >> (2 * p)) & 1u, i1 = (v >> (2 * p + 1)) & 1u;
-          o[p] = __byte_perm(c0, c0, 0x1010u + i0 * 0x22u + i1 * 0x2200u);
+          for (int i = 0; i < 8; ++i) v |= ((u >> field_pos<2>(i, true)) & 3u) << (2 * i);
+        } else {
+          // field 2c' at bit 15 - c', field 2c'+1 at bit 31 - c'; chunk q holds c' = 4q .. 4q+3
+          const uint32_t u = t << (4 * q);
+          v = 0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) v |= ((u >> field_pos<1>(i, true)) & 1u) << i;
         }
+      } else if constexpr (BITS == 4) {
+        v = __ldg(row_words + c);
       } else if constexpr (BITS == 2) {
-        // codebook = 8 bytes {c0,c1 | c2,c3}: byte pair (2i, 2i+1) of the two words
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-          const uint32_t i0 = (v >> (4 * p)) & 3u, i1 = (v >> (4 * p + 2)) & 3u;
-          o[p] = __byte_perm(c0, c1, 0x1010u + i0 * 0x22u + i1 * 0x2200u);
-        }
+        v = __ldg(reinterpret_cast<const uint16_t*>(row_words) + c);
       } else {
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-          const uint32_t i0 = (v >> (8 * p)) & 15u, i1 = (v >> (8 * p + 4)) & 15u;
-          o[p] = (uint32_t)__ldg(row_cb + i0) | ((uint32_t)__ldg(row_cb + i1) << 16);
-        }
+        v = __ldg(reinterpret_cast<const uint8_t*>(row_words) + c);
       }
-      stg_stream_u4(out + c, make_uint4(o[0], o[1], o[2], o[3]));
+      stg_stream_u4(out + c, decode8<BITS>(v, c0, c1, row_cb));
     }
   }
 }
@@ -96,16 +103,16 @@ cudaError_t launch_dequant(const uint32_t* packed, const uint16_t* cb, uint16_t*
                            int layout, cudaStream_t s) {
   const DeviceInfo* di = device_info();
   if (!di) return cudaGetLastError();
+  const bool tuned = layout == KMQ_LAYOUT_TUNED;
   int64_t blocks = N;
   const int64_t cap = (int64_t)di->sm_count * 8;   // 8 resident CTAs of 256 threads per SM
   if (blocks > cap) blocks = cap;
-  const bool tuned = layout == KMQ_LAYOUT_TUNED;
-  if (bits == 1 && tuned) dequant_kernel<1, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
-  else if (bits == 1) dequant_kernel<1, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
-  else if (bits == 2 && tuned) dequant_kernel<2, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
-  else if (bits == 2) dequant_kernel<2, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
-  else if (tuned) dequant_kernel<4, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
-  else dequant_kernel<4, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  if (bits == 1 && tuned) dequant_rows_kernel<1, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  else if (bits == 1) dequant_rows_kernel<1, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  else if (bits == 2 && tuned) dequant_rows_kernel<2, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  else if (bits == 2) dequant_rows_kernel<2, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  else if (tuned) dequant_rows_kernel<4, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+  else dequant_rows_kernel<4, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
   return cudaGetLastError();
 }
 
