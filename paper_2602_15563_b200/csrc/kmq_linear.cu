@@ -12,6 +12,15 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
     const bool tuned = layout == KMQ_LAYOUT_TUNED;
     p.variant = tuned ? kVariantTiled : kVariantMma;
     p.launches = (int)((M + 7) / 8);
+    // b = 4 with at most 16 rows: two passes of the GEMV kernel (pair tables, 2 weights per lookup) beat the
+    // single-entry tables of the multi-tile kernel, whose decode is shared by only 2 MMAs there
+    if (tuned && M > 8 && !(bits == 4 && M <= 16)) {
+      const int64_t per = linear_multi_rows_per_launch(bits);
+      p.variant = kVariantMulti;
+      p.launches = (int)((M + per - 1) / per);
+      p.name = bits == 4 ? "multi_table_b4" : bits == 2 ? "multi_prmt_b2" : "multi_sign_b1";
+      return p;
+    }
     if (bits == 4) p.name = tuned ? "tiled_pairtable_b4" : "staged_pairtable_b4";
     else if (bits == 2) p.name = tuned ? "tiled_prmt_b2" : "staged_prmt_b2";
     else p.name = tuned ? "tiled_sign_b1" : "staged_sign_b1";
@@ -28,6 +37,8 @@ cudaError_t launch_linear(const LinearPlan& plan, const uint32_t* packed, const 
                           cudaStream_t s) {
   (void)workspace;
   switch (plan.variant) {
+    case kVariantMulti:
+      return launch_linear_multi(packed, cb, x, y, N, K, bits, M, s);
     case kVariantTiled:
       return launch_linear_tiled(packed, cb, x, y, N, K, bits, M, s);
     case kVariantMma:

@@ -1,0 +1,334 @@
+// kmq_linear on the tuned (tile-major) layout for batches of 9..64 rows: the decode of a weight fragment is paid
+// once and reused by up to 8 MMAs (one per group of 8 batch rows).
+//
+// One CTA owns 64 output rows = 4 tiles.  Its 8 warps are 2 K-groups of 4 warps; warp (group, i) owns tile i and the
+// steps s = group, group + 2, ... of it.  The 4 warps of a K-group walk the same steps together and share the
+// activations under a step: they are copied global -> shared with cp.async, double buffered, one named barrier per
+// step.  Per step a warp decodes its 1 KB of packed indices (two 128-bit loads issued one step earlier) into
+// mma.sync.m16n8k16 A fragments and multiplies each fragment with the NT B fragments (batch rows 8 nt .. 8 nt + 7)
+// read from shared memory.  At the end the second K-group hands its accumulators to the first through shared
+// memory, which adds them, applies the b = 1 codebook and stores bf16.
+//
+// b = 4 uses single-entry per-row tables here (16 entries x 32 lane banks, 4 KB per tile; one LDS per weight and a
+// PRMT per pair): the 64 KB pair tables of the GEMV kernel would not fit for 4 tiles, and the decode is amortised
+// over NT MMAs anyway.
+#include "kmq_common.cuh"
+#include "kmq_linear_variants.cuh"
+#include "kmq_mma_common.cuh"
+
+namespace kmq {
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kTilesPerCta = 4;
+constexpr int kGroups = 2;
+constexpr int kGroupThreads = 128;
+constexpr int kTableBytesPerTile = 2 * 16 * 32 * 4;   // b = 4: [half][entry][lane] words
+
+template <int BITS>
+struct MGeo {
+  static constexpr int kMmaPerWord = 8 / BITS;
+  static constexpr int kStepK = 512 / BITS;
+  static constexpr int kWordK = 32 / BITS;
+  static constexpr int kChunkXBytes = 4 * kWordK * 2;     // activations under one 16-byte chunk of a row
+  static constexpr int kChunkStride = kChunkXBytes + 16;  // +16 bytes: conflict-free 16-byte B-fragment loads
+  static constexpr int kRowStride = 4 * kChunkStride;     // one batch row of one step
+  static constexpr int kPiecesPerRow = kStepK / 8;        // 16-byte pieces per batch row and step
+  static constexpr int kTableBytes = BITS == 4 ? kTilesPerCta * kTableBytesPerTile : 0;
+};
+
+template <int BITS, int NT>
+struct MSmem {
+  using G = MGeo<BITS>;
+  static constexpr int kBuf = 8 * NT * G::kRowStride;            // one x buffer: 8 NT batch rows of one step
+  static constexpr int kX = kGroups * 2 * kBuf;                  // double buffered, per K-group
+  static constexpr int kRed = kTilesPerCta * 32 * NT * 4 * 4;    // accumulators of the second K-group (aliases x)
+  static constexpr int kSums = kGroups * 8 * NT * 4;             // b = 1: sum of x per batch row and K-group
+  static constexpr int kTotal = G::kTableBytes + (kX > kRed ? kX : kRed) + kSums;
+};
+
+template <int BITS>
+__device__ __forceinline__ int piece_offset(int w) {
+  using G = MGeo<BITS>;
+  constexpr int kPiecesPerChunk = G::kChunkXBytes / 16;
+  return (w / kPiecesPerChunk) * G::kChunkStride + (w % kPiecesPerChunk) * 16;
+}
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, bool valid) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  const int bytes = valid ? 16 : 0;   // 0 source bytes: the 16 destination bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gmem_src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void group_barrier(int group) {
+  asm volatile("bar.sync %0, %1;" ::"r"(group + 1), "r"(kGroupThreads) : "memory");
+}
+
+template <int BITS, int NT>
+__global__ void __launch_bounds__(kThreads, 1) linear_multi_kernel(const uint32_t* __restrict__ packed,
+                                                                    const uint16_t* __restrict__ cb,
+                                                                    const uint16_t* __restrict__ x,
+                                                                    uint16_t* __restrict__ y, int64_t N, int64_t K,
+                                                                    int M) {
+  using G = MGeo<BITS>;
+  using SM = MSmem<BITS, NT>;
+  constexpr int Q = G::kMmaPerWord;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  unsigned char* const tables = smem_raw;
+  unsigned char* const xbase = smem_raw + G::kTableBytes;
+  float* const red = reinterpret_cast<float*>(xbase);                       // reused after the main loop
+  float* const sums = reinterpret_cast<float*>(xbase + (SM::kX > SM::kRed ? SM::kX : SM::kRed));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int wt = warp & 3, group = warp >> 2;          // tile inside the CTA, K-group
+  const int gtid = threadIdx.x & (kGroupThreads - 1);  // thread inside the K-group
+  const int64_t tiles = (N + kTileRows - 1) / kTileRows;
+  const int64_t tile_id = (int64_t)blockIdx.x * kTilesPerCta + wt;
+  const bool has_tile = tile_id < tiles;               // warp-uniform; such a warp still stages x and joins barriers
+  const int64_t row0 = tile_id * kTileRows;
+  const int chunks = (int)(K / (4 * G::kWordK));
+  const int steps = (chunks + 3) >> 2;
+  const uint4* __restrict__ tile =
+      reinterpret_cast<const uint4*>(packed) + (has_tile ? tile_id : 0) * (int64_t)steps * 64 + lane;
+  unsigned char* const xgroup = xbase + group * 2 * SM::kBuf;
+
+  // copy the activations under step s into buffer `buf` of this K-group (zeros past K; rows >= M are not touched:
+  // their MMA columns are never stored)
+  auto stage = [&](int s, int buf) {
+    unsigned char* dst = xgroup + buf * SM::kBuf;
+    const int total = M * G::kPiecesPerRow;
+    for (int p = gtid; p < total; p += kGroupThreads) {
+      const int m = p / G::kPiecesPerRow, w = p % G::kPiecesPerRow;
+      const int64_t k = (int64_t)s * G::kStepK + w * 8;
+      const bool ok = k < K;
+      cp_async16(dst + m * G::kRowStride + piece_offset<BITS>(w), x + (int64_t)m * K + (ok ? k : 0), ok);
+    }
+    cp_async_commit();
+  };
+
+  // ---- first loads: weights of this warp's first two steps, activations of the group's first step ----
+  uint4 qa[2], qb[2];
+#pragma unroll
+  for (int d = 0; d < 2; ++d) {
+    const int s = group + d * kGroups;
+    qa[d] = qb[d] = make_uint4(0, 0, 0, 0);
+    if (has_tile && s < steps) {
+      qa[d] = ldg_stream_u4(tile + (int64_t)s * 64);
+      qb[d] = ldg_stream_u4(tile + (int64_t)s * 64 + 32);
+    }
+  }
+  if (group < steps) stage(group, 0);
+
+  // ---- per-row decode state ----
+  Dec2 dg, dh;
+  if constexpr (BITS == 2) {
+    dg.init(cb + min(row0 + g, N - 1) * 4);
+    dh.init(cb + min(row0 + g + 8, N - 1) * 4);
+  }
+  if constexpr (BITS == 4) {
+    // word (tile, half, entry e, lane) = C_row[e] in both halves, row = 16 tile + 8 half + lane / 4
+    for (int i = threadIdx.x; i < kTilesPerCta * 2 * 16 * 32; i += kThreads) {
+      const int ln = i & 31, e = (i >> 5) & 15, half = (i >> 9) & 1, tl = i >> 10;
+      const int64_t r = min(((int64_t)blockIdx.x * kTilesPerCta + tl) * kTileRows + 8 * half + (ln >> 2), N - 1);
+      const uint32_t c = __ldg(cb + r * 16 + e);
+      reinterpret_cast<uint32_t*>(tables)[i] = c | (c << 16);
+    }
+    __syncthreads();
+  }
+  const unsigned char* const tab_g = tables + wt * kTableBytesPerTile;   // rows g; rows g + 8 are 2 KB further
+  const uint32_t lane4 = lane * 4;
+
+  float acc[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+  // b = 1: warp wt of a K-group sums the activations of batch rows m = wt, wt + 4, ... (2 NT of them)
+  float sacc[2 * NT];
+#pragma unroll
+  for (int i = 0; i < 2 * NT; ++i) sacc[i] = 0.f;
+
+  for (int s0 = group; s0 < steps; s0 += 2 * kGroups) {   // uniform over the K-group
+#pragma unroll
+   for (int buf = 0; buf < 2; ++buf) {                     // buffer index = parity of the group's step count
+    const int s = s0 + buf * kGroups;
+    if (s >= steps) break;
+    cp_async_wait_all();
+    group_barrier(group);   // x of step s is in place, and every warp of the group is done with step s - 2
+    if (s + kGroups < steps) stage(s + kGroups, buf ^ 1);
+    const unsigned char* const xs = xgroup + buf * SM::kBuf;
+    if (has_tile) {
+      const uint4 va = qa[buf], vb = qb[buf];
+      const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
+      const uint32_t wb[4] = {vb.x, vb.y, vb.z, vb.w};
+      if (s + 2 * kGroups < steps) {   // refill for the step after next
+        qa[buf] = ldg_stream_u4(tile + (int64_t)(s + 2 * kGroups) * 64);
+        qb[buf] = ldg_stream_u4(tile + (int64_t)(s + 2 * kGroups) * 64 + 32);
+      }
+      const unsigned char* const xb = xs + g * G::kRowStride + t * G::kChunkStride;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int q2 = 0; q2 < Q; q2 += 2) {
+          uint4 xv[NT];   // 16 bytes of x per batch row = the k-slots of two consecutive MMAs
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+            xv[nt] = *reinterpret_cast<const uint4*>(xb + nt * 8 * G::kRowStride + (j * Q + q2) * 8);
+#pragma unroll
+          for (int qq = 0; qq < 2; ++qq) {
+            const int q = q2 + qq;
+            uint32_t a0, a1, a2, a3;
+            if constexpr (BITS == 2) {
+              dg.pair(wa[j], q, a0, a2);
+              dh.pair(wb[j], q, a1, a3);
+            } else if constexpr (BITS == 4) {
+              // nibbles 4q .. 4q+3 of the word: weights (4q, 4q+1 | 4q+2, 4q+3); offset = (nibble << 7) | lane * 4
+              uint32_t lo[4], hi[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int sh = 4 * (4 * q + i) - 7;
+                const uint32_t ua = sh < 0 ? (wa[j] << -sh) : (wa[j] >> sh);
+                const uint32_t ub = sh < 0 ? (wb[j] << -sh) : (wb[j] >> sh);
+                lo[i] = *reinterpret_cast<const uint32_t*>(tab_g + and_or(ua, 0x780u, lane4));
+                hi[i] = *reinterpret_cast<const uint32_t*>(tab_g + 2048 + and_or(ub, 0x780u, lane4));
+              }
+              a0 = prmt(lo[0], lo[1], 0x7610u);
+              a2 = prmt(lo[2], lo[3], 0x7610u);
+              a1 = prmt(hi[0], hi[1], 0x7610u);
+              a3 = prmt(hi[2], hi[3], 0x7610u);
+            } else {
+              const uint32_t m0 = kPow2[2 * q], m1 = kPow2[2 * q + 1];
+              a0 = and_or(wa[j] * m0, 0x80008000u, 0x3F803F80u);
+              a2 = and_or(wa[j] * m1, 0x80008000u, 0x3F803F80u);
+              a1 = and_or(wb[j] * m0, 0x80008000u, 0x3F803F80u);
+              a3 = and_or(wb[j] * m1, 0x80008000u, 0x3F803F80u);
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+              mma_bf16_16816(acc[nt], a0, a1, a2, a3, qq ? xv[nt].z : xv[nt].x, qq ? xv[nt].w : xv[nt].y);
+          }
+        }
+      }
+    }
+    if constexpr (BITS == 1) {
+      // S[m] = sum_k x[m,k]: the 512 staged activations of a batch row as two 16x16 A tiles times ones
+#pragma unroll
+      for (int i = 0; i < 2 * NT; ++i) {
+        const int m = wt + 4 * i;
+        if (m < M) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const uint4 v = *reinterpret_cast<const uint4*>(xs + m * G::kRowStride + piece_offset<BITS>(lane + 32 * h));
+            float tmp[4] = {0.f, 0.f, 0.f, 0.f};
+            mma_bf16_16816(tmp, v.x, v.y, v.z, v.w, 0x3F803F80u, 0x3F803F80u);
+            sacc[i] += tmp[0] + tmp[2];
+          }
+        }
+      }
+    }
+   }
+  }
+
+  // ---- K-group 1 hands its partial sums to K-group 0, which adds, applies the codebook (b = 1) and stores ----
+  if constexpr (BITS == 1) {
+#pragma unroll
+    for (int i = 0; i < 2 * NT; ++i) {
+      float v = sacc[i];
+      v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
+      v += __shfl_xor_sync(0xFFFFFFFFu, v, 8);
+      v += __shfl_xor_sync(0xFFFFFFFFu, v, 16);
+      if (lane == 0) sums[group * 8 * NT + wt + 4 * i] = v;   // lanes with t = 0 cover every row once
+    }
+  }
+  __syncthreads();   // every warp is done with the x buffers; `red` aliases them
+  if (group == 1) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+      *reinterpret_cast<float4*>(red + ((wt * NT + nt) * 32 + lane) * 4) =
+          make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
+  }
+  __syncthreads();
+  if (group == 0 && has_tile) {
+    uint32_t cw0 = 0, cw1 = 0;
+    if constexpr (BITS == 1) {
+      cw0 = __ldg(reinterpret_cast<const uint32_t*>(cb + min(row0 + g, N - 1) * 2));
+      cw1 = __ldg(reinterpret_cast<const uint32_t*>(cb + min(row0 + g + 8, N - 1) * 2));
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float4 o = *reinterpret_cast<const float4*>(red + ((wt * NT + nt) * 32 + lane) * 4);
+      const float v[4] = {acc[nt][0] + o.x, acc[nt][1] + o.y, acc[nt][2] + o.z, acc[nt][3] + o.w};
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int m = nt * 8 + 2 * t + (r & 1);
+        const int64_t n = row0 + g + 8 * (r >> 1);
+        if (m < M && n < N) {
+          float out = v[r];
+          if constexpr (BITS == 1) {
+            const float sx = sums[m] + sums[8 * NT + m];
+            const uint32_t c = (r >> 1) ? cw1 : cw0;
+            const float c0 = bf16_bits_to_float(c & 0xFFFFu), c1 = bf16_bits_to_float(c >> 16);
+            out = fmaf(c0, 0.5f * (sx + out), c1 * (0.5f * (sx - out)));
+          }
+          y[(int64_t)m * N + n] = (uint16_t)float_to_bf16_bits(out);
+        }
+      }
+    }
+  }
+}
+
+template <int BITS, int NT>
+cudaError_t launch_nt(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N, int64_t K,
+                      int M, cudaStream_t s) {
+  constexpr int smem = MSmem<BITS, NT>::kTotal;
+  static bool configured[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    cudaError_t e =
+        cudaFuncSetAttribute(linear_multi_kernel<BITS, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  const int64_t tiles = (N + kTileRows - 1) / kTileRows;
+  const unsigned grid = (unsigned)((tiles + kTilesPerCta - 1) / kTilesPerCta);
+  linear_multi_kernel<BITS, NT><<<grid, kThreads, smem, s>>>(packed, cb, x, y, N, K, M);
+  return cudaGetLastError();
+}
+
+template <int BITS>
+cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                        int64_t K, int M, cudaStream_t s) {
+  if (M <= 16) return launch_nt<BITS, 2>(packed, cb, x, y, N, K, M, s);
+  if (M <= 32) return launch_nt<BITS, 4>(packed, cb, x, y, N, K, M, s);
+  if constexpr (BITS == 1) {
+    return cudaErrorInvalidValue;   // unreachable: b = 1 is launched in passes of at most 32 rows
+  } else {
+    return launch_nt<BITS, 8>(packed, cb, x, y, N, K, M, s);
+  }
+}
+
+}  // namespace
+
+// Batch rows per launch of the multi-tile kernel: 64, or 32 for b = 1 (its x buffers are twice as large).
+int linear_multi_rows_per_launch(int bits) { return bits == 1 ? 32 : 64; }
+
+cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                                int64_t K, int bits, int64_t M, cudaStream_t s) {
+  const int64_t per = linear_multi_rows_per_launch(bits);
+  for (int64_t m0 = 0; m0 < M; m0 += per) {
+    const int mc = (int)(M - m0 < per ? M - m0 : per);
+    const uint16_t* xp = x + m0 * K;
+    uint16_t* yp = y + m0 * N;
+    cudaError_t e;
+    if (mc <= 8) e = launch_linear_tiled(packed, cb, xp, yp, N, K, bits, mc, s);   // a short tail
+    else if (bits == 1) e = launch_bits<1>(packed, cb, xp, yp, N, K, mc, s);
+    else if (bits == 2) e = launch_bits<2>(packed, cb, xp, yp, N, K, mc, s);
+    else e = launch_bits<4>(packed, cb, xp, yp, N, K, mc, s);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace kmq

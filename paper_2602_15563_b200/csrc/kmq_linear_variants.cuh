@@ -7,7 +7,8 @@ namespace kmq {
 enum LinearVariant : int {
   kVariantGeneric = 0,   // any legal shape and layout, CUDA-core FMAs, one warp per output row
   kVariantMma = 1,       // canonical layout, K*bits % 128 == 0: tensor-core GEMV, activations staged per warp
-  kVariantTiled = 2,     // tuned (tile-major) layout: tensor-core GEMV with coalesced 1 KB steps
+  kVariantTiled = 2,     // tuned (tile-major) layout: tensor-core GEMV with coalesced 1 KB steps, M <= 8
+  kVariantMulti = 3,     // tuned layout, M > 8: 64 rows per CTA, one decode feeds up to 8 MMAs
 };
 
 cudaError_t launch_linear_generic(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
@@ -17,6 +18,10 @@ bool linear_mma_supports(int64_t N, int64_t K, int bits, int64_t M);
 cudaError_t launch_linear_mma(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                               int64_t K, int bits, int64_t M, cudaStream_t s);
 cudaError_t launch_linear_tiled(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                                int64_t K, int bits, int64_t M, cudaStream_t s);
+
+int linear_multi_rows_per_launch(int bits);
+cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                 int64_t K, int bits, int64_t M, cudaStream_t s);
 
 }  // namespace kmq
