@@ -12,9 +12,7 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
     const bool tuned = layout == KMQ_LAYOUT_TUNED;
     p.variant = tuned ? kVariantTiled : kVariantMma;
     p.launches = (int)((M + 7) / 8);
-    // b = 4 with at most 16 rows: two passes of the GEMV kernel (pair tables, 2 weights per lookup) beat the
-    // single-entry tables of the multi-tile kernel, whose decode is shared by only 2 MMAs there
-    if (tuned && M > 8 && !(bits == 4 && M <= 16)) {
+    if (tuned && M > 8) {
       const int64_t per = linear_multi_rows_per_launch(bits);
       p.variant = kVariantMulti;
       p.launches = (int)((M + per - 1) / per);

@@ -123,6 +123,12 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
     }
   }
 
+  // b = 1: the codebook is only needed by the epilogue, but fetching it there would add a memory round trip
+  uint32_t cb1 = 0;
+  if constexpr (BITS == 1) {
+    if (threadIdx.x < kRows * 8) cb1 = __ldg(reinterpret_cast<const uint32_t*>(cb + min(row0 + (threadIdx.x & 15), N - 1) * 2));
+  }
+
   // ---- per-row decode state ----
   Dec2 dg, dh;
   if constexpr (BITS == 2) {
@@ -130,12 +136,19 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
     dh.init(cb + min(row0 + g + 8, N - 1) * 4);
   }
   if constexpr (BITS == 4) {
-    // entry e of row r: (C_r[e & 15], C_r[e >> 4]); the 4 lanes that share a row get one bank each
-    const int r8 = threadIdx.x & 7, half = (threadIdx.x >> 3) & 1;
+    // entry e of row r: (C_r[e & 15], C_r[e >> 4]); the 4 lanes that share a row get one bank each.
+    // A thread owns one row and one low index: it fetches the row's 16 centroids once (32 bytes) and writes the
+    // 16 entries e = low + 16 * high with no further loads.
+    const int r8 = threadIdx.x & 7, half = (threadIdx.x >> 3) & 1, low = threadIdx.x >> 4;
     const uint16_t* crow = cb + min(row0 + r8 + 8 * half, N - 1) * 16;
-    for (int e = threadIdx.x >> 4; e < 256; e += kThreads / 16) {
-      const uint32_t v = (uint32_t)__ldg(crow + (e & 15)) | ((uint32_t)__ldg(crow + (e >> 4)) << 16);
-      *reinterpret_cast<uint4*>(tables + e * kPairEntryStride + half * 128 + r8 * 16) = make_uint4(v, v, v, v);
+    const uint4 ca = __ldg(reinterpret_cast<const uint4*>(crow)), cc = __ldg(reinterpret_cast<const uint4*>(crow) + 1);
+    const uint32_t lo = __ldg(crow + low);
+    const uint32_t c2[8] = {ca.x, ca.y, ca.z, ca.w, cc.x, cc.y, cc.z, cc.w};
+    unsigned char* dst = tables + low * kPairEntryStride + half * 128 + r8 * 16;
+#pragma unroll
+    for (int hi = 0; hi < 16; ++hi) {
+      const uint32_t v = prmt(lo, c2[hi >> 1], (hi & 1) ? 0x7610u : 0x5410u);   // (C[low], C[hi])
+      *reinterpret_cast<uint4*>(dst + hi * 16 * kPairEntryStride) = make_uint4(v, v, v, v);
     }
     __syncthreads();
   }
@@ -252,8 +265,7 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) sx += red_s[w * MMAX + mm];
         // v = T0 - T1, sx = T0 + T1 with T_i the sum of the activations whose weight has index i
-        const uint32_t c = __ldg(reinterpret_cast<const uint32_t*>(cb + n * 2));
-        const float c0 = bf16_bits_to_float(c & 0xFFFFu), c1 = bf16_bits_to_float(c >> 16);
+        const float c0 = bf16_bits_to_float(cb1 & 0xFFFFu), c1 = bf16_bits_to_float(cb1 >> 16);
         v = fmaf(c0, 0.5f * (sx + v), c1 * (0.5f * (sx - v)));
       }
       y[(int64_t)m * N + n] = (uint16_t)float_to_bf16_bits(v);
