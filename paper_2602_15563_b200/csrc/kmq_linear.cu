@@ -19,6 +19,17 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
       p.name = bits == 4 ? "multi_table_b4" : bits == 2 ? "multi_prmt_b2" : "multi_sign_b1";
       return p;
     }
+    if (tuned) {
+      const int ctas = linear_split_ctas(N, K, bits, M);
+      if (ctas > 0) {
+        p.variant = kVariantSplit;
+        p.launches = 2;
+        p.split_k = ctas;
+        p.workspace = linear_split_scratch_bytes(ctas);
+        p.name = bits == 4 ? "split_pairtable_b4" : bits == 2 ? "split_prmt_b2" : "split_sign_b1";
+        return p;
+      }
+    }
     if (bits == 4) p.name = tuned ? "tiled_pairtable_b4" : "staged_pairtable_b4";
     else if (bits == 2) p.name = tuned ? "tiled_prmt_b2" : "staged_prmt_b2";
     else p.name = tuned ? "tiled_sign_b1" : "staged_sign_b1";
@@ -33,8 +44,9 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
 cudaError_t launch_linear(const LinearPlan& plan, const uint32_t* packed, const uint16_t* cb, const uint16_t* x,
                           uint16_t* y, int64_t N, int64_t K, int bits, int64_t M, int layout, void* workspace,
                           cudaStream_t s) {
-  (void)workspace;
   switch (plan.variant) {
+    case kVariantSplit:
+      return launch_linear_split(packed, cb, x, y, N, K, bits, M, workspace, plan.split_k, s);
     case kVariantMulti:
       return launch_linear_multi(packed, cb, x, y, N, K, bits, M, s);
     case kVariantTiled:

@@ -58,12 +58,13 @@ __device__ __forceinline__ int piece_offset(int w) {
   return (w / kPiecesPerChunk) * G::kChunkStride + (w % kPiecesPerChunk) * 16;
 }
 
+// Steps [sa, sb) of tile `tile_id`, all 8 warps of the CTA: on return thread i < 128 holds in `v` the sum over those
+// steps for output row i % 16 and batch row i / 16 (b = 1: the signed sum D, and in `sx` the sum of the activations
+// under those steps).  May be called several times by one CTA; shared memory is reused from call to call.
 template <int BITS, int MMAX>
-__global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_t* __restrict__ packed,
-                                                                    const uint16_t* __restrict__ cb,
-                                                                    const uint16_t* __restrict__ x,
-                                                                    uint16_t* __restrict__ y, int64_t N, int64_t K,
-                                                                    int M) {
+__device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed, const uint16_t* __restrict__ cb,
+                                             const uint16_t* __restrict__ x, int64_t N, int64_t K, int M,
+                                             int64_t tile_id, int sa, int sb, float& v, float& sx) {
   using G = TGeo<BITS>;
   using SM = TSmem<BITS, MMAX>;
   constexpr int Q = G::kMmaPerWord;
@@ -81,11 +82,12 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int64_t row0 = (int64_t)blockIdx.x * kRows;
+  const int64_t row0 = tile_id * kRows;
   const int chunks = (int)(K / (4 * G::kWordK));   // 16-byte chunks per row
   const int steps = (chunks + 3) >> 2;             // the layout pads every row to whole steps
   // step s of this tile: 64 16-byte units, unit h * 32 + lane = row (g + 8h), chunk t
-  const uint4* __restrict__ tile = reinterpret_cast<const uint4*>(packed) + (int64_t)blockIdx.x * steps * 64 + lane;
+  const uint4* __restrict__ tile = reinterpret_cast<const uint4*>(packed) + tile_id * steps * 64 + lane;
+  __syncthreads();   // a previous segment's readers of the tables and of `red` are done
 
   // ---- x pieces of this lane: piece p = lane + 32 i -> batch row p / kPiecesPerRow, piece p % kPiecesPerRow
   int px_k[NP], px_sm[NP];
@@ -112,21 +114,15 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
   uint4 qa[STAGES], qb[STAGES], qx[XS][NP];
 #pragma unroll
   for (int d = 0; d < STAGES; ++d) {
-    const int s = warp + d * kWarps;
+    const int s = sa + warp + d * kWarps;
     qa[d] = qb[d] = make_uint4(0, 0, 0, 0);
 #pragma unroll
     for (int i = 0; i < NP; ++i) qx[kPrefetchX ? d : 0][i] = make_uint4(0, 0, 0, 0);
-    if (s < steps) {
+    if (s < sb) {
       qa[d] = ldg_stream_u4(tile + (int64_t)s * 64);
       qb[d] = ldg_stream_u4(tile + (int64_t)s * 64 + 32);
       if constexpr (kPrefetchX) load_x(s, qx[kPrefetchX ? d : 0]);
     }
-  }
-
-  // b = 1: the codebook is only needed by the epilogue, but fetching it there would add a memory round trip
-  uint32_t cb1 = 0;
-  if constexpr (BITS == 1) {
-    if (threadIdx.x < kRows * 8) cb1 = __ldg(reinterpret_cast<const uint32_t*>(cb + min(row0 + (threadIdx.x & 15), N - 1) * 2));
   }
 
   // ---- per-row decode state ----
@@ -163,11 +159,11 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
   // g >= M re-read the last real row and their columns are never stored.
   const unsigned char* const xb = xs_warp + min(g, M - 1) * G::kRowStride + t * G::kChunkStride;
 
-  for (int s0 = warp; s0 < steps; s0 += STAGES * kWarps) {
+  for (int s0 = sa + warp; s0 < sb; s0 += STAGES * kWarps) {
 #pragma unroll
     for (int d = 0; d < STAGES; ++d) {
       const int s = s0 + d * kWarps;
-      if (s < steps) {   // warp-uniform
+      if (s < sb) {   // warp-uniform
         // stage the activations under this step (zeros past K)
         if constexpr (!kPrefetchX) load_x(s, qx[0]);
         __syncwarp();
@@ -229,7 +225,7 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
         }
         // refill this stage for the step kStages rounds ahead
         const int s2 = s + STAGES * kWarps;
-        if (s2 < steps) {
+        if (s2 < sb) {
           qa[d] = ldg_stream_u4(tile + (int64_t)s2 * 64);
           qb[d] = ldg_stream_u4(tile + (int64_t)s2 * 64 + 32);
           if constexpr (kPrefetchX) load_x(s2, qx[kPrefetchX ? d : 0]);
@@ -251,19 +247,31 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
     }
   }
   __syncthreads();
+  v = 0.f;
+  sx = 0.f;
   if (threadIdx.x < kRows * 8) {
     const int r = threadIdx.x & 15, m = threadIdx.x >> 4;   // consecutive threads -> consecutive output rows
+    const int src_lane = (r & 7) * 4 + (m >> 1), src_reg = (r >> 3) * 2 + (m & 1);
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) v += red[(w * 32 + src_lane) * 4 + src_reg];
+    if constexpr (BITS == 1) {
+      const int mm = m < MMAX ? m : 0;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) sx += red_s[w * MMAX + mm];
+    }
+  }
+}
+
+// Thread i < 128: apply the codebook (b = 1) to the finished sum of output row row0 + i % 16, batch row i / 16, and
+// store it as bf16.  `cb1` = the two centroids of that row (b = 1 only).
+template <int BITS>
+__device__ __forceinline__ void store_output(float v, float sx, uint32_t cb1, uint16_t* __restrict__ y, int64_t N,
+                                             int M, int64_t row0) {
+  if (threadIdx.x < kRows * 8) {
+    const int r = threadIdx.x & 15, m = threadIdx.x >> 4;
     const int64_t n = row0 + r;
     if (m < M && n < N) {
-      const int src_lane = (r & 7) * 4 + (m >> 1), src_reg = (r >> 3) * 2 + (m & 1);
-      float v = 0.f;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) v += red[(w * 32 + src_lane) * 4 + src_reg];
       if constexpr (BITS == 1) {
-        float sx = 0.f;
-        const int mm = m < MMAX ? m : 0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) sx += red_s[w * MMAX + mm];
         // v = T0 - T1, sx = T0 + T1 with T_i the sum of the activations whose weight has index i
         const float c0 = bf16_bits_to_float(cb1 & 0xFFFFu), c1 = bf16_bits_to_float(cb1 >> 16);
         v = fmaf(c0, 0.5f * (sx + v), c1 * (0.5f * (sx - v)));
@@ -271,6 +279,85 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
       y[(int64_t)m * N + n] = (uint16_t)float_to_bf16_bits(v);
     }
   }
+}
+
+// b = 1: the two centroids of the output row thread i < 128 will store; fetched early, off the critical path.
+template <int BITS>
+__device__ __forceinline__ uint32_t load_cb1(const uint16_t* __restrict__ cb, int64_t N, int64_t row0) {
+  if constexpr (BITS == 1) {
+    if (threadIdx.x < kRows * 8)
+      return __ldg(reinterpret_cast<const uint32_t*>(cb + min(row0 + (threadIdx.x & 15), N - 1) * 2));
+  }
+  return 0;
+}
+
+// One CTA per tile.
+template <int BITS, int MMAX>
+__global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_t* __restrict__ packed,
+                                                                    const uint16_t* __restrict__ cb,
+                                                                    const uint16_t* __restrict__ x,
+                                                                    uint16_t* __restrict__ y, int64_t N, int64_t K,
+                                                                    int M) {
+  const int steps = (int)((K / (4 * TGeo<BITS>::kWordK) + 3) >> 2);
+  const int64_t row0 = (int64_t)blockIdx.x * kRows;
+  const uint32_t cb1 = load_cb1<BITS>(cb, N, row0);
+  float v, sx;
+  tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, blockIdx.x, 0, steps, v, sx);
+  store_output<BITS>(v, sx, cb1, y, N, M, row0);
+}
+
+// ---------------------------------------------------------------------------
+// Balanced variant for more tiles than resident CTA slots.  The tiles * steps step-units, in tile-major order, are
+// cut into gridDim.x equal contiguous ranges, one per CTA (all CTAs resident at once, so no second wave).  A range
+// is longer than a tile, so a CTA finishes the tiles that lie wholly inside its range and owns at most two partial
+// tiles, one at each end; their sums go to scratch slot [cta][0] (range starts inside the tile) or [cta][1] (range
+// ends inside it).  Every cut therefore has exactly two contributors, which the fix-up kernel adds in a fixed order.
+// ---------------------------------------------------------------------------
+constexpr int kSlotFloats = kRows * 8 + 8;   // 128 sums + 8 sums of x (b = 1)
+
+template <int BITS, int MMAX>
+__global__ void __launch_bounds__(kThreads, 3) linear_split_kernel(const uint32_t* __restrict__ packed,
+                                                                    const uint16_t* __restrict__ cb,
+                                                                    const uint16_t* __restrict__ x,
+                                                                    uint16_t* __restrict__ y, int64_t N, int64_t K,
+                                                                    int M, float* __restrict__ scratch) {
+  const int64_t steps = (K / (4 * TGeo<BITS>::kWordK) + 3) >> 2;
+  const int64_t units = ((N + kRows - 1) / kRows) * steps;
+  const int64_t u0 = units * blockIdx.x / gridDim.x, u1 = units * (blockIdx.x + 1) / gridDim.x;
+  for (int64_t tile = u0 / steps; tile * steps < u1; ++tile) {
+    const int64_t base = tile * steps;
+    const int sa = (int)(u0 > base ? u0 - base : 0), sb = (int)(u1 - base < steps ? u1 - base : steps);
+    const uint32_t cb1 = load_cb1<BITS>(cb, N, tile * kRows);
+    float v, sx;
+    tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, tile, sa, sb, v, sx);
+    if (sa == 0 && sb == steps) {
+      store_output<BITS>(v, sx, cb1, y, N, M, tile * kRows);
+    } else if (threadIdx.x < kRows * 8) {
+      float* slot = scratch + ((int64_t)blockIdx.x * 2 + (sa == 0 ? 1 : 0)) * kSlotFloats;
+      slot[threadIdx.x] = v;
+      if (BITS == 1 && (threadIdx.x & 15) == 0) slot[kRows * 8 + (threadIdx.x >> 4)] = sx;
+    }
+  }
+}
+
+// Block c adds the two halves of the tile that the cut between CTA c and CTA c + 1 falls into.
+template <int BITS>
+__global__ void __launch_bounds__(kRows * 8) linear_split_fixup_kernel(const float* __restrict__ scratch,
+                                                                       const uint16_t* __restrict__ cb,
+                                                                       uint16_t* __restrict__ y, int64_t N, int64_t K,
+                                                                       int M, int ctas) {
+  const int64_t steps = (K / (4 * TGeo<BITS>::kWordK) + 3) >> 2;
+  const int64_t units = ((N + kRows - 1) / kRows) * steps;
+  const int64_t cut = units * (blockIdx.x + 1) / ctas;
+  if (cut % steps == 0) return;   // the cut is a tile boundary: nothing was left partial
+  const int64_t row0 = (cut / steps) * kRows;
+  const float* end_of_c = scratch + ((int64_t)blockIdx.x * 2 + 1) * kSlotFloats;
+  const float* start_of_next = scratch + ((int64_t)(blockIdx.x + 1) * 2) * kSlotFloats;
+  const int m = threadIdx.x >> 4;
+  const float v = end_of_c[threadIdx.x] + start_of_next[threadIdx.x];
+  float sx = 0.f;
+  if constexpr (BITS == 1) sx = end_of_c[kRows * 8 + m] + start_of_next[kRows * 8 + m];
+  store_output<BITS>(v, sx, load_cb1<BITS>(cb, N, row0), y, N, M, row0);
 }
 
 template <int BITS, int MMAX>
@@ -300,6 +387,35 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
   return launch_one<BITS, 8>(packed, cb, x, y, N, K, M, s);
 }
 
+template <int BITS, int MMAX>
+cudaError_t launch_split_one(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                             int64_t K, int M, float* scratch, int ctas, cudaStream_t s) {
+  constexpr int smem = TSmem<BITS, MMAX>::kTotal;
+  static bool configured[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    cudaError_t e =
+        cudaFuncSetAttribute(linear_split_kernel<BITS, MMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  linear_split_kernel<BITS, MMAX><<<ctas, kThreads, smem, s>>>(packed, cb, x, y, N, K, M, scratch);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  linear_split_fixup_kernel<BITS><<<ctas - 1, kRows * 8, 0, s>>>(scratch, cb, y, N, K, M, ctas);
+  return cudaGetLastError();
+}
+
+template <int BITS>
+cudaError_t launch_split_bits(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                              int64_t K, int M, float* scratch, int ctas, cudaStream_t s) {
+  if (M == 1) return launch_split_one<BITS, 1>(packed, cb, x, y, N, K, M, scratch, ctas, s);
+  if (M == 2) return launch_split_one<BITS, 2>(packed, cb, x, y, N, K, M, scratch, ctas, s);
+  if (M <= 4) return launch_split_one<BITS, 4>(packed, cb, x, y, N, K, M, scratch, ctas, s);
+  return launch_split_one<BITS, 8>(packed, cb, x, y, N, K, M, scratch, ctas, s);
+}
+
 }  // namespace
 
 // Tuned layout.  Batches larger than 8 are processed 8 rows at a time (one launch each).
@@ -316,6 +432,35 @@ cudaError_t launch_linear_tiled(const uint32_t* packed, const uint16_t* cb, cons
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
+}
+
+}  // namespace kmq
+
+namespace kmq {
+
+// CTAs of the balanced variant (0 = use one CTA per tile): all resident slots when there are more tiles than slots.
+// Every range restarts the load pipeline and the decode set-up once or twice more than a whole tile would, so this
+// only pays when a tile is long: at least kSplitMinSteps steps (measured: 8192 x 28672, b = 4, 224 steps, 55 -> 44 us;
+// with 16..56 steps per tile the per-tile grid is faster).
+constexpr int64_t kSplitMinSteps = 128;
+
+int linear_split_ctas(int64_t N, int64_t K, int bits, int64_t M) {
+  const DeviceInfo* di = device_info();
+  if (!di || M > 8) return 0;
+  const int64_t slots = (int64_t)di->sm_count * 3;
+  const int64_t tiles = (N + kRows - 1) / kRows;
+  const int64_t steps = (K * bits / 128 + 3) / 4;
+  return (tiles > slots && steps >= kSplitMinSteps) ? (int)slots : 0;
+}
+
+size_t linear_split_scratch_bytes(int ctas) { return (size_t)ctas * 2 * kSlotFloats * sizeof(float); }
+
+cudaError_t launch_linear_split(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                                int64_t K, int bits, int64_t M, void* scratch, int ctas, cudaStream_t s) {
+  float* sc = static_cast<float*>(scratch);
+  if (bits == 1) return launch_split_bits<1>(packed, cb, x, y, N, K, (int)M, sc, ctas, s);
+  if (bits == 2) return launch_split_bits<2>(packed, cb, x, y, N, K, (int)M, sc, ctas, s);
+  return launch_split_bits<4>(packed, cb, x, y, N, K, (int)M, sc, ctas, s);
 }
 
 }  // namespace kmq

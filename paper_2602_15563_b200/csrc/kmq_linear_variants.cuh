@@ -9,6 +9,7 @@ enum LinearVariant : int {
   kVariantMma = 1,       // canonical layout, K*bits % 128 == 0: tensor-core GEMV, activations staged per warp
   kVariantTiled = 2,     // tuned (tile-major) layout: tensor-core GEMV with coalesced 1 KB steps, M <= 8
   kVariantMulti = 3,     // tuned layout, M > 8: 64 rows per CTA, one decode feeds up to 8 MMAs
+  kVariantSplit = 4,     // tuned layout, M <= 8, more tiles than resident CTAs: equal step ranges + fix-up (scratch)
 };
 
 cudaError_t launch_linear_generic(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
@@ -20,6 +21,10 @@ cudaError_t launch_linear_mma(const uint32_t* packed, const uint16_t* cb, const 
 cudaError_t launch_linear_tiled(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                 int64_t K, int bits, int64_t M, cudaStream_t s);
 
+int linear_split_ctas(int64_t N, int64_t K, int bits, int64_t M);
+size_t linear_split_scratch_bytes(int ctas);
+cudaError_t launch_linear_split(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                                int64_t K, int bits, int64_t M, void* scratch, int ctas, cudaStream_t s);
 int linear_multi_rows_per_launch(int bits);
 cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                 int64_t K, int bits, int64_t M, cudaStream_t s);

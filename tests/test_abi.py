@@ -53,7 +53,9 @@ def test_sizes_and_strings():
     assert kmq.kmq_packed_bytes(4096, 4096, 2, layout=T) == 4096 * 4096 // 4      # whole tiles and steps: no padding
     assert kmq.kmq_packed_bytes(17, 32, 1, layout=T) == 2 * 1 * 1024               # 2 tiles x 1 step x 1 KB
     assert kmq.kmq_packed_bytes(16, 8 * 17, 4, layout=T) == 1 * 2 * 1024            # 17 words per row -> 2 steps
-    assert kmq.kmq_linear_num_launches(4096, 4096, 2, 17, layout=T) == 3
+    assert kmq.kmq_linear_num_launches(4096, 4096, 2, 17) == 3                    # canonical: passes of 8 batch rows
+    assert kmq.kmq_linear_num_launches(4096, 4096, 2, 17, layout=T) == 1          # tuned: one multi-tile launch
+    assert kmq.kmq_linear_num_launches(4096, 4096, 1, 64, layout=T) == 2          # b = 1: 32 batch rows per launch
     assert kmq.kmq_linear_variant(4096, 4096, 2, 1, layout=7) == "invalid"
     assert kmq.kmq_linear_variant(4096, 4096, 2, 1, layout=T) != kmq.kmq_linear_variant(4096, 4096, 2, 1)
 

@@ -154,13 +154,33 @@ def test_host_entry_point_matches_device_entry_point():
 
 
 def test_workspace_is_checked_on_the_host():
-    N, K, bits, M = 3072, 8192, 2, 1
-    need = kmq.kmq_workspace_bytes(N, K, bits, M)
+    N, K, bits, M, T = 8192, 16384, 4, 1, kmq.KMQ_LAYOUT_TUNED
+    need = kmq.kmq_workspace_bytes(N, K, bits, M, T)
     if need == 0:
-        pytest.skip("this shape needs no workspace")
+        pytest.skip("this shape needs no workspace on this device")
     a = torch.zeros(16, dtype=torch.uint8, device="cuda")
     big = torch.zeros(N * K // 4, dtype=torch.uint8, device="cuda")
-    st = kmq.kmq_linear(big, big, big, big, N, K, bits, M, a, need - 1, check=False)
+    st = kmq.kmq_linear(big, big, big, big, N, K, bits, M, a, need - 1, layout=T, check=False)
     assert st == kmq.KMQ_ERR_WORKSPACE
-    st = kmq.kmq_linear(big, big, big, big, N, K, bits, M, None, 0, check=False)
+    st = kmq.kmq_linear(big, big, big, big, N, K, bits, M, None, 0, layout=T, check=False)
     assert st == kmq.KMQ_ERR_WORKSPACE
+
+
+# ---- more tiles than resident CTAs: equal step ranges per CTA, partial tiles added by the fix-up kernel ----
+@pytest.mark.parametrize("bits", BITS)
+@pytest.mark.parametrize("Kmul,M", [(512, 1), (517, 8)])
+def test_linear_balanced_split_variant(bits, Kmul, M):
+    N, K = 16 * 460 + 5, (128 // bits) * Kmul          # 461 tiles (the last one ragged), Kmul 16-byte chunks per row
+    rng = np.random.default_rng(7000 + 10 * bits + Kmul)
+    idx, cb, x = random_layer(rng, N, K, bits, M)
+    T = kmq.KMQ_LAYOUT_TUNED
+    if kmq.kmq_workspace_bytes(N, K, bits, M, T) == 0:
+        pytest.skip("the balanced variant is not selected on this device")
+    assert kmq.kmq_linear_num_launches(N, K, bits, M, T) == 2
+    ref_packed = orc.pack_canonical(idx, bits)
+    y_ref, s = orc.linear_f64(ref_packed, cb, x, K, bits)
+    packed = gu.gpu_pack(idx, bits, T)
+    y1 = gu.gpu_linear(packed, cb, x, N, K, bits, T)
+    ratio = orc.check_linear(y1, y_ref, s)
+    assert ratio <= 1.0, f"error/tolerance = {ratio} [{kmq.kmq_linear_variant(N, K, bits, M, T)}]"
+    assert np.array_equal(y1, gu.gpu_linear(packed, cb, x, N, K, bits, T)), "repeated call differs"
