@@ -63,7 +63,8 @@ typedef enum {
   KMQ_ERR_ALIGN = 4,     /* a device pointer is not 16-byte aligned */
   KMQ_ERR_WORKSPACE = 5, /* workspace missing or smaller than kmq_workspace_bytes() */
   KMQ_ERR_LAYOUT = 6,    /* unknown layout id */
-  KMQ_ERR_CUDA = 7       /* the CUDA runtime reported an error (launch, copy) */
+  KMQ_ERR_CUDA = 7,      /* the CUDA runtime reported an error (launch, copy) */
+  KMQ_ERR_SCRATCH_LIMIT = 8 /* kmq_linear_static_scratch: the shape needs more than the built-in scratch holds */
 } kmq_status;
 
 typedef enum {
@@ -135,6 +136,31 @@ kmq_status kmq_linear_host(const uint32_t* packed, const uint16_t* codebooks, co
                            uint16_t* y_host, int64_t N, int64_t K, int bits, int64_t M, int layout,
                            uint16_t* x_dev, uint16_t* y_dev, void* workspace, size_t workspace_bytes,
                            void* stream);
+
+/*
+ * kmq_linear_static_scratch -- kmq_linear without a workspace argument, for
+ * callers that are not allowed to allocate device memory: code inside a region
+ * where the allocator must not be entered (a latency-critical loop, a
+ * non-blocking callback), or a component that owns nothing but the buffers it
+ * was given.  (This is a convenience of this library; the paper has no
+ * counterpart.)  Same arguments, result and errors as kmq_linear.  Where
+ * kmq_linear would need scratch (kmq_workspace_bytes() > 0) the partial sums
+ * go to a fixed 512 KiB array that is part of the library image on every GPU
+ * that loads it (kmq_static_scratch_capacity() returns the size); a shape that
+ * needs more is refused with KMQ_ERR_SCRATCH_LIMIT and nothing is launched.
+ * The call never allocates or frees memory.
+ *   - The first call on each device looks up the array's device address
+ *     (once, with that device current); make that first call outside any
+ *     stream capture.
+ *   - All calls on a device share the one array.  Calls whose kernels may
+ *     overlap on the GPU (different streams, or graph branches) race on it:
+ *     serialise them.  Its contents between calls are meaningless and never
+ *     need clearing: each call writes every word it later reads.
+ */
+kmq_status kmq_linear_static_scratch(const uint32_t* packed, const uint16_t* codebooks,
+                                     const uint16_t* x, uint16_t* y, int64_t N, int64_t K, int bits,
+                                     int64_t M, int layout, void* stream);
+size_t kmq_static_scratch_capacity(void);
 
 /*
  * kmq_dequant_to_bf16 -- materialise W^[n,k] = C_n[idx[n,k]] as a dense bf16

@@ -57,6 +57,7 @@ const char* kmq_status_string(int status) {
     case KMQ_ERR_WORKSPACE: return "workspace missing or too small";
     case KMQ_ERR_LAYOUT: return "unknown packed layout";
     case KMQ_ERR_CUDA: return "CUDA runtime error";
+    case KMQ_ERR_SCRATCH_LIMIT: return "the shape needs more scratch than the built-in static buffer holds";
     default: return "unknown status";
   }
 }

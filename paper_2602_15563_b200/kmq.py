@@ -17,6 +17,7 @@ _lib = None
 KMQ_OK = 0
 KMQ_ERR_NULL, KMQ_ERR_BITS, KMQ_ERR_SHAPE, KMQ_ERR_ALIGN = 1, 2, 3, 4
 KMQ_ERR_WORKSPACE, KMQ_ERR_LAYOUT, KMQ_ERR_CUDA = 5, 6, 7
+KMQ_ERR_SCRATCH_LIMIT = 8
 KMQ_LAYOUT_CANONICAL = 0
 KMQ_LAYOUT_TUNED = 1
 
@@ -34,6 +35,8 @@ SIGNATURES = {
     "kmq_unpack": (_int, [_ptr, _i64, _i64, _int, _int, _ptr, _ptr]),
     "kmq_linear": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr, _sz, _ptr]),
     "kmq_linear_host": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr, _ptr, _ptr, _sz, _ptr]),
+    "kmq_linear_static_scratch": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr]),
+    "kmq_static_scratch_capacity": (_sz, []),
     "kmq_dequant_to_bf16": (_int, [_ptr, _ptr, _ptr, _i64, _i64, _int, _int, _ptr]),
 }
 
@@ -140,6 +143,20 @@ def kmq_linear_host(packed, codebooks, x_host, y_host, N, K, bits, M, x_dev, y_d
     if check:
         _check(st, "kmq_linear_host")
     return st
+
+
+def kmq_linear_static_scratch(packed, codebooks, x, y, N, K, bits, M, layout=KMQ_LAYOUT_CANONICAL, stream=None,
+                              check=True) -> int:
+    """kmq_linear for callers that may not allocate: scratch, where needed, is a fixed array inside the library."""
+    st = lib().kmq_linear_static_scratch(_addr(packed), _addr(codebooks), _addr(x), _addr(y), N, K, bits, M, layout,
+                                         _stream(stream))
+    if check:
+        _check(st, "kmq_linear_static_scratch")
+    return st
+
+
+def kmq_static_scratch_capacity() -> int:
+    return lib().kmq_static_scratch_capacity()
 
 
 def kmq_dequant_to_bf16(packed, codebooks, W, N, K, bits, layout=KMQ_LAYOUT_CANONICAL, stream=None, check=True) -> int:
