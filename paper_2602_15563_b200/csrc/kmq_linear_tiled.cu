@@ -27,6 +27,9 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kRows = kTileRows;
 constexpr int kPairEntryStride = 256;   // b = 4 tables: entry e, half h, lane l at e * 256 + h * 128 + l * 4
 constexpr int kTableBytes4 = 256 * kPairEntryStride;
+#ifndef KMQ_PDL
+#define KMQ_PDL 1
+#endif
 
 template <int BITS>
 struct TGeo {
@@ -298,11 +301,20 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
                                                                     const uint16_t* __restrict__ x,
                                                                     uint16_t* __restrict__ y, int64_t N, int64_t K,
                                                                     int M) {
+#if KMQ_PDL
+  // Programmatic dependent launch: nothing is read before the previous kernel on the stream has completed (same
+  // ordering as a plain launch), but this grid could be set up while that kernel drained, and the next kernel may be
+  // set up while this one sums and stores.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
   const int steps = (int)((K / (4 * TGeo<BITS>::kWordK) + 3) >> 2);
   const int64_t row0 = (int64_t)blockIdx.x * kRows;
   const uint32_t cb1 = load_cb1<BITS>(cb, N, row0);
   float v, sx;
   tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, blockIdx.x, 0, steps, v, sx);
+#if KMQ_PDL
+  asm volatile("griddepcontrol.launch_dependents;");
+#endif
   store_output<BITS>(v, sx, cb1, y, N, M, row0);
 }
 
@@ -373,9 +385,17 @@ cudaError_t launch_one(const uint32_t* packed, const uint16_t* cb, const uint16_
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  const unsigned grid = (unsigned)((N + kRows - 1) / kRows);
-  linear_tiled_kernel<BITS, MMAX><<<grid, kThreads, smem, s>>>(packed, cb, x, y, N, K, M);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((N + kRows - 1) / kRows));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = KMQ_PDL ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, linear_tiled_kernel<BITS, MMAX>, packed, cb, x, y, N, K, M);
 }
 
 template <int BITS>
