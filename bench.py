@@ -43,7 +43,8 @@ WORKLOADS = {
     "config3_m8": [(n, N, K, "student_t", 2, 8) for n, N, K in
                    (("qkv", 9216, 3072), ("o", 3072, 3072), ("gate_up", 16384, 3072), ("down", 3072, 8192))],
     "config4": [("square8192", 8192, 8192, "normal", 2, m) for m in (1, 2, 4, 8, 16, 32, 64)],
-    "config5": [("down_large", 8192, 28672, "laplace", b, m) for b in (1, 4) for m in (1, 16)],
+    "config5": [("down_large", 8192, 28672, "laplace", b, m) for b in (1, 4) for m in (1, 16)] +
+               [("down_large", 8192, 28672, "laplace", b, 0) for b in (1, 4)],     # M = 0: kmq_dequant_to_bf16
     "tiny": [("tiny", 256, 256, "normal", b, 1) for b in (1, 2, 4)],
 }
 WORKLOAD_TEXT = {
@@ -53,7 +54,8 @@ WORKLOAD_TEXT = {
                   "down 8192->3072), b=2, batch 1, Student-t(5) weights",
     "config3_m8": "3.9B-style decoder linear set, b=2, batch 8, Student-t(5) weights",
     "config4": "batch sweep on N=K=8192, b=2, batch in {1,2,4,8,16,32,64}",
-    "config5": "large down projection N=8192 K=28672, b in {1,4}, batch in {1,16}, Laplace weights",
+    "config5": "large down projection N=8192 K=28672, b in {1,4}, batch in {1,16}, Laplace weights, plus the "
+               "standalone kmq_dequant_to_bf16 of the full matrix (cases with M=0)",
     "tiny": "256x256 correctness layer",
 }
 CONFIG_ID = {"config2": 2, "config3_m1": 3, "config3_m8": 3, "config4": 4, "config5": 5, "tiny": 1}
@@ -64,7 +66,20 @@ NCU_TRAFFIC_BYTES = {}
 
 
 def algorithmic_bytes(N, K, bits, M):
+    if M == 0:                                   # kmq_dequant_to_bf16: packed + codebooks read, dense bf16 written
+        return N * K * bits // 8 + N * (1 << bits) * 2 + 2 * N * K
     return N * K * bits // 8 + N * (1 << bits) * 2 + M * K * 2 + M * N * 2
+
+
+_LAYER_CACHE = {}
+
+
+def cached_layer(synth, N, K, bits, dist, config_id):
+    """Weights, codebooks and indices depend on (shape, bits, distribution) only: fit them once per process."""
+    key = (N, K, bits, dist, config_id)
+    if key not in _LAYER_CACHE:
+        _LAYER_CACHE[key] = synth.make_layer(N, K, bits, 1, dist, config_id=config_id)
+    return _LAYER_CACHE[key]
 
 
 def measured_peak():
@@ -138,35 +153,48 @@ class Case:
         self.name, self.N, self.K, self.bits, self.M = name, N, K, bits, M
         self.bytes = algorithmic_bytes(N, K, bits, M)
         self.pool = max(4, -(-pool_bytes // self.bytes))
-        layer = synth.make_layer(N, K, bits, M, dist, config_id=config_id)
+        layer = dict(cached_layer(synth, N, K, bits, dist, config_id))
+        self.dequant = M == 0
+        rng = synth.rng_for(config_id, 100 + bits * 1000 + M)
+        layer["x"] = synth.draw_activations(max(M, 1), K, synth.rng_for(config_id, synth.TENSOR_X))
         self.layer = layer
         dev = torch.device("cuda")
         idx = torch.from_numpy(layer["idx"]).to(dev)
         self.layout = kmq.KMQ_LAYOUT_TUNED                         # the layout the fast kernels read
         words = kmq.kmq_packed_bytes(N, K, bits, self.layout) // 4
+        if self.dequant:
+            self.pool = max(2, -(-pool_bytes // self.bytes))
         self.packed = torch.empty((self.pool, words), dtype=torch.int32, device=dev)
         kmq.kmq_pack(idx, N, K, bits, self.packed[0], layout=self.layout)   # a1: offline packing, on the GPU
         self.packed[1:] = self.packed[0]
         del idx
         cb = torch.from_numpy(layer["codebooks"].view(np.int16)).to(dev)
         self.cb = cb.unsqueeze(0).repeat(self.pool, 1, 1).contiguous()
-        rng = synth.rng_for(config_id, 100 + bits * 1000 + M)
-        xs = np.stack([layer["x"]] + [synth.draw_activations(M, K, rng) for _ in range(self.pool - 1)])
+        Mx = max(M, 1)
+        xs = np.stack([layer["x"]] + [synth.draw_activations(Mx, K, rng) for _ in range(self.pool - 1)])
         self.x_host = torch.from_numpy(xs.view(np.int16)).pin_memory()
         self.x = self.x_host.to(dev)
-        self.y = torch.zeros((self.pool, M, N), dtype=torch.int16, device=dev)
-        self.y_host = torch.zeros((self.pool, M, N), dtype=torch.int16).pin_memory()
-        self.ws_bytes = kmq.kmq_workspace_bytes(N, K, bits, M, self.layout)
+        if self.dequant:
+            self.W = torch.zeros((self.pool, N, K), dtype=torch.int16, device=dev)
+        self.y = torch.zeros((self.pool, Mx, N), dtype=torch.int16, device=dev)
+        self.y_host = torch.zeros((self.pool, Mx, N), dtype=torch.int16).pin_memory()
+        self.ws_bytes = 0 if self.dequant else kmq.kmq_workspace_bytes(N, K, bits, M, self.layout)
         self.ws = torch.empty(max(self.ws_bytes, 16), dtype=torch.uint8, device=dev)
-        self.launches = kmq.kmq_linear_num_launches(N, K, bits, M, self.layout)
-        self.variant = kmq.kmq_linear_variant(N, K, bits, M, self.layout)
+        self.launches = 1 if self.dequant else kmq.kmq_linear_num_launches(N, K, bits, M, self.layout)
+        self.variant = "dequant_rows" if self.dequant else kmq.kmq_linear_variant(N, K, bits, M, self.layout)
         self.kmq = kmq
 
     def call(self, i):
+        if self.dequant:
+            self.kmq.kmq_dequant_to_bf16(self.packed[i], self.cb[i], self.W[i], self.N, self.K, self.bits,
+                                         layout=self.layout)
+            return
         self.kmq.kmq_linear(self.packed[i], self.cb[i], self.x[i], self.y[i], self.N, self.K, self.bits, self.M,
                             self.ws, self.ws_bytes, layout=self.layout)
 
     def call_host(self, i):
+        if self.dequant:                         # nothing to copy in or out: the weights stay on the device
+            return self.call(i)
         self.kmq.kmq_linear_host(self.packed[i], self.cb[i], self.x_host[i].data_ptr(), self.y_host[i].data_ptr(),
                                  self.N, self.K, self.bits, self.M, self.x[i], self.y[i], self.ws, self.ws_bytes,
                                  layout=self.layout)
@@ -293,18 +321,27 @@ def run_library(args):
             dist.destroy_process_group()
         return
 
-    # ---- parity spot check of what was just timed (rank 0) ----
+    # ---- parity spot check of what was just timed (rank 0): sampled output rows against the oracle ----
     from oracle import kmq_oracle as orc
     worst = 0.0
     checked = 0
     for c in cases:
-        ref_packed = orc.pack_canonical(c.layer["idx"], c.bits)
+        rows = np.unique(np.concatenate([np.arange(16), np.arange(c.N - 16, c.N),
+                                         np.random.default_rng(c.bits + c.M).choice(c.N, 32, replace=False)]))
+        ref_packed = orc.pack_canonical(c.layer["idx"][rows], c.bits)
+        cb_rows = c.layer["codebooks"][rows]
+        d_rows = torch.from_numpy(rows).cuda()
         for i in sorted({0, c.pool - 1}):
-            x_i = c.x_host[i].numpy().view(np.uint16)
-            y_ref, s = orc.linear_f64(ref_packed, c.layer["codebooks"], x_i, c.K, c.bits)
-            y = c.y[i].cpu().numpy().view(np.uint16)
-            yh = c.y_host[i].numpy().view(np.uint16)
-            worst = max(worst, orc.check_linear(y, y_ref, s), orc.check_linear(yh, y_ref, s))
+            if c.dequant:
+                got = c.W[i][d_rows].cpu().numpy().view(np.uint16)
+                ok = np.array_equal(got, orc.dequant_bits(ref_packed, cb_rows, c.K, c.bits))
+                worst = max(worst, 0.0 if ok else float("inf"))
+            else:
+                x_i = c.x_host[i].numpy().view(np.uint16)
+                y_ref, s = orc.linear_f64(ref_packed, cb_rows, x_i, c.K, c.bits)
+                y = c.y[i][:, d_rows].cpu().numpy().view(np.uint16)
+                yh = c.y_host[i].numpy().view(np.uint16)[:, rows]
+                worst = max(worst, orc.check_linear(y, y_ref, s), orc.check_linear(yh, y_ref, s))
             checked += 1
 
     # ---- per-case figures and the roofline of the dominant kernel ----
@@ -365,37 +402,53 @@ def _cpu_threads():
         return len(os.sched_getaffinity(0))
 
 
+ORACLE_MAX_WEIGHTS = 1 << 24     # per oracle call: larger layers are timed on their first rows only
+
+
 def _oracle_cases(workload):
+    """(N_sample, K, bits, M, packed rows, codebook rows, x, bytes of the sample) per case of the workload."""
     from oracle import kmq_oracle as orc
     from paper_2602_15563_b200 import synth
     out = []
     for (name, N, K, d, b, M) in WORKLOADS[workload]:
-        layer = synth.make_layer(N, K, b, M, d, config_id=CONFIG_ID[workload])
-        out.append((N, K, b, M, orc.pack_canonical(layer["idx"], b), layer["codebooks"], layer["x"]))
+        layer = cached_layer(synth, N, K, b, d, CONFIG_ID[workload])
+        n = int(min(N, max(16, ORACLE_MAX_WEIGHTS // K)))
+        x = synth.draw_activations(max(M, 1), K, synth.rng_for(CONFIG_ID[workload], synth.TENSOR_X))
+        out.append((n, K, b, M, orc.pack_canonical(layer["idx"][:n], b), layer["codebooks"][:n], x,
+                    algorithmic_bytes(n, K, b, M)))
     return out
 
 
+def _oracle_call(orc, case):
+    n, K, b, M, packed, cb, x, _bytes = case
+    if M == 0:
+        orc.dequant_bits(packed, cb, K, b)
+    else:
+        orc.linear_f64(packed, cb, x, K, b)
+
+
 def cpu_baseline(workload, budget_s=12.0, cases=None):
-    """Time the oracle's inference part (unpack, table lookup, float64 matmul)
-    on the host cores, on a bounded sample of the workload."""
+    """Time the oracle's inference part (unpack, table lookup, float64 matmul) on the host cores, on a bounded
+    sample of the workload: every case once per pass, layers larger than ORACLE_MAX_WEIGHTS cut to their first rows."""
     from oracle import kmq_oracle as orc
     cases = cases or _oracle_cases(workload)
-    for (N, K, b, M, packed, cb, x) in cases[:1]:
-        orc.linear_f64(packed, cb, x, K, b)                       # warm-up
+    _oracle_call(orc, cases[0])                                   # warm-up
     total_bytes, n_calls = 0, 0
     t0 = time.perf_counter()
     while True:
-        for (N, K, b, M, packed, cb, x) in cases:
-            orc.linear_f64(packed, cb, x, K, b)
-            total_bytes += algorithmic_bytes(N, K, b, M)
+        for case in cases:
+            _oracle_call(orc, case)
+            total_bytes += case[7]
             n_calls += 1
         if time.perf_counter() - t0 >= budget_s or n_calls >= 1000:
             break
     dt = time.perf_counter() - t0
+    rows = sorted({c[0] for c in cases})
     return {"value": round(total_bytes / dt / 1e9, 4), "unit": "GB/s", "cores": _cpu_threads(),
             "host_cores": len(os.sched_getaffinity(0)), "kind": "oracle",
             "sample": f"{n_calls} oracle calls ({n_calls // len(cases)} pass(es) over the {len(cases)} cases of "
-                      f"{workload}, one weight set each), {dt:.1f} s", "us_per_call": round(dt / n_calls * 1e6, 1)}
+                      f"{workload}, one weight set each, first {rows} rows of each layer), {dt:.1f} s",
+            "us_per_call": round(dt / n_calls * 1e6, 1)}
 
 
 def run_reference(args):
@@ -405,11 +458,11 @@ def run_reference(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     from oracle import kmq_oracle as orc
     cases = _oracle_cases(args.workload)
-    step_bytes = sum(algorithmic_bytes(N, K, b, M) for (N, K, b, M, *_r) in cases)
+    step_bytes = sum(c[7] for c in cases)
 
     def step():
-        for (N, K, b, M, packed, cb, x) in cases:
-            orc.linear_f64(packed, cb, x, K, b)
+        for case in cases:
+            _oracle_call(orc, case)
 
     steps = max(1, min(args.steps, 40))
     for _ in range(max(1, min(args.warmup, 3))):
@@ -420,7 +473,8 @@ def run_reference(args):
     dt = time.perf_counter() - t0
     value = step_bytes * steps / dt / 1e9
     cores = _cpu_threads()
-    sample = f"one oracle call per case of {args.workload} per step ({len(cases)} calls), {steps} steps"
+    sample = (f"one oracle call per case of {args.workload} per step ({len(cases)} calls, first "
+              f"{sorted({c[0] for c in cases})} rows of each layer), {steps} steps")
     line = {
         "impl": "reference",
         "metric": "kmq_linear effective HBM bandwidth (algorithmic bytes / time), batch-1 k-means LUT GEMV",
