@@ -82,6 +82,13 @@ const char* kmq_status_string(int status);
  * tile-major size (tuned); 0 if the arguments are invalid. */
 size_t kmq_packed_bytes(int64_t N, int64_t K, int bits, int layout);
 
+/* Where the packed layouts put things (host-side arithmetic, no GPU involved):
+ * kmq_packed_word_index -- index, in 32-bit words from the start of the packed
+ * buffer, of word j of row n; kmq_packed_field_shift -- bit position of field i
+ * (index idx[n, j*(32/bits) + i]) inside that word.  -1 for invalid arguments. */
+int64_t kmq_packed_word_index(int64_t n, int64_t j, int64_t N, int64_t K, int bits, int layout);
+int kmq_packed_field_shift(int i, int bits, int layout);
+
 /* Bytes of scratch kmq_linear needs for this shape on the current device
  * (fp32 partial sums of a split along K); may be 0. */
 size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M, int layout);

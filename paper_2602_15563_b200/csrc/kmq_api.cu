@@ -69,6 +69,19 @@ size_t kmq_packed_bytes(int64_t N, int64_t K, int bits, int layout) {
   return (size_t)N * (size_t)wpr * 4u;
 }
 
+int64_t kmq_packed_word_index(int64_t n, int64_t j, int64_t N, int64_t K, int bits, int layout) {
+  if (!known_layout(layout) || check_shape(N, K, bits, 1) != KMQ_OK) return -1;
+  const int64_t wpr = K / (32 / bits);
+  if (n < 0 || n >= N || j < 0 || j >= wpr) return -1;
+  return layout == KMQ_LAYOUT_TUNED ? tuned_word_index(n, j, tuned_steps(wpr)) : n * wpr + j;
+}
+
+int kmq_packed_field_shift(int i, int bits, int layout) {
+  if (!known_layout(layout) || (bits != 1 && bits != 2 && bits != 4) || i < 0 || i >= 32 / bits) return -1;
+  const bool tuned = layout == KMQ_LAYOUT_TUNED;
+  return bits == 1 ? field_pos<1>(i, tuned) : bits == 2 ? field_pos<2>(i, tuned) : field_pos<4>(i, tuned);
+}
+
 size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M, int layout) {
   if (!known_layout(layout) || check_shape(N, K, bits, M) != KMQ_OK) return 0;
   return plan_linear(N, K, bits, M, layout).workspace;

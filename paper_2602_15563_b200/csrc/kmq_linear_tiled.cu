@@ -22,7 +22,16 @@
 namespace kmq {
 namespace {
 
-constexpr int kWarps = 8;
+#ifndef KMQ_TILED_WARPS
+#define KMQ_TILED_WARPS 8
+#endif
+#ifndef KMQ_TILED_MINB
+#define KMQ_TILED_MINB 3
+#endif
+#ifndef KMQ_TILED_STAGES4
+#define KMQ_TILED_STAGES4 2
+#endif
+constexpr int kWarps = KMQ_TILED_WARPS;
 constexpr int kThreads = kWarps * 32;
 constexpr int kRows = kTileRows;
 constexpr int kPairEntryStride = 256;   // b = 4 tables: entry e, half h, lane l at e * 256 + h * 128 + l * 4
@@ -41,7 +50,7 @@ struct TGeo {
   static constexpr int kRowStride = 4 * kChunkStride;     // one batch row of one step
   static constexpr int kPiecesPerRow = kStepK / 8;        // 16-byte pieces of x per batch row and step
   static constexpr int kTableBytes = BITS == 4 ? kTableBytes4 : 0;
-  static constexpr int kStages = BITS == 4 ? 4 : 2;       // steps in flight per warp
+  static constexpr int kStages = BITS == 4 ? KMQ_TILED_STAGES4 : 2;       // steps in flight per warp (deeper rings measured slower)
 };
 
 template <int BITS, int MMAX>
@@ -138,7 +147,9 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
     // entry e of row r: (C_r[e & 15], C_r[e >> 4]); the 4 lanes that share a row get one bank each.
     // A thread owns one row and one low index: it fetches the row's 16 centroids once (32 bytes) and writes the
     // 16 entries e = low + 16 * high with no further loads.
-    const int r8 = threadIdx.x & 7, half = (threadIdx.x >> 3) & 1, low = threadIdx.x >> 4;
+    const int r8 = threadIdx.x & 7, half = (threadIdx.x >> 3) & 1, low = (threadIdx.x >> 4) & 15;
+    constexpr int kParts = kThreads / 256;   // threads beyond the first 256 take a share of the high indices
+    const int part = threadIdx.x >> 8;
     const uint16_t* crow = cb + min(row0 + r8 + 8 * half, N - 1) * 16;
     const uint4 ca = __ldg(reinterpret_cast<const uint4*>(crow)), cc = __ldg(reinterpret_cast<const uint4*>(crow) + 1);
     const uint32_t lo = __ldg(crow + low);
@@ -146,6 +157,7 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
     unsigned char* dst = tables + low * kPairEntryStride + half * 128 + r8 * 16;
 #pragma unroll
     for (int hi = 0; hi < 16; ++hi) {
+      if (kParts > 1 && (hi % kParts) != part) continue;
       const uint32_t v = prmt(lo, c2[hi >> 1], (hi & 1) ? 0x7610u : 0x5410u);   // (C[low], C[hi])
       *reinterpret_cast<uint4*>(dst + hi * 16 * kPairEntryStride) = make_uint4(v, v, v, v);
     }
@@ -296,7 +308,7 @@ __device__ __forceinline__ uint32_t load_cb1(const uint16_t* __restrict__ cb, in
 
 // One CTA per tile.
 template <int BITS, int MMAX>
-__global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_t* __restrict__ packed,
+__global__ void __launch_bounds__(kThreads, KMQ_TILED_MINB) linear_tiled_kernel(const uint32_t* __restrict__ packed,
                                                                     const uint16_t* __restrict__ cb,
                                                                     const uint16_t* __restrict__ x,
                                                                     uint16_t* __restrict__ y, int64_t N, int64_t K,
@@ -328,7 +340,7 @@ __global__ void __launch_bounds__(kThreads, 3) linear_tiled_kernel(const uint32_
 constexpr int kSlotFloats = kRows * 8 + 8;   // 128 sums + 8 sums of x (b = 1)
 
 template <int BITS, int MMAX>
-__global__ void __launch_bounds__(kThreads, 3) linear_split_kernel(const uint32_t* __restrict__ packed,
+__global__ void __launch_bounds__(kThreads, KMQ_TILED_MINB) linear_split_kernel(const uint32_t* __restrict__ packed,
                                                                     const uint16_t* __restrict__ cb,
                                                                     const uint16_t* __restrict__ x,
                                                                     uint16_t* __restrict__ y, int64_t N, int64_t K,

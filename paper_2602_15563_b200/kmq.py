@@ -28,6 +28,8 @@ SIGNATURES = {
     "kmq_version": (_int, []),
     "kmq_status_string": (ctypes.c_char_p, [_int]),
     "kmq_packed_bytes": (_sz, [_i64, _i64, _int, _int]),
+    "kmq_packed_word_index": (_i64, [_i64, _i64, _i64, _i64, _int, _int]),
+    "kmq_packed_field_shift": (_int, [_int, _int, _int]),
     "kmq_workspace_bytes": (_sz, [_i64, _i64, _int, _i64, _int]),
     "kmq_linear_num_launches": (_int, [_i64, _i64, _int, _i64, _int]),
     "kmq_linear_variant": (ctypes.c_char_p, [_i64, _i64, _int, _i64, _int]),
@@ -95,6 +97,14 @@ def kmq_version() -> int:
 
 def kmq_packed_bytes(N, K, bits, layout=KMQ_LAYOUT_CANONICAL) -> int:
     return lib().kmq_packed_bytes(N, K, bits, layout)
+
+
+def kmq_packed_word_index(n, j, N, K, bits, layout=KMQ_LAYOUT_CANONICAL) -> int:
+    return lib().kmq_packed_word_index(n, j, N, K, bits, layout)
+
+
+def kmq_packed_field_shift(i, bits, layout=KMQ_LAYOUT_CANONICAL) -> int:
+    return lib().kmq_packed_field_shift(i, bits, layout)
 
 
 def kmq_workspace_bytes(N, K, bits, M, layout=KMQ_LAYOUT_CANONICAL) -> int:

@@ -77,3 +77,26 @@ def gpu_linear(packed: torch.Tensor, cb: np.ndarray, x: np.ndarray, N: int, K: i
     assert canaries_intact(buf, off, nbytes), "linear wrote outside y"
     assert canaries_intact(wsbuf, wsoff, max(ws_bytes, 16)), "linear wrote outside its workspace"
     return buf[off:off + nbytes].cpu().numpy().view(np.uint16).reshape(M, N)
+
+
+def tuned_from_canonical(words: np.ndarray, bits: int) -> np.ndarray:
+    """The documented tuned layout (include/kmq.h) applied to canonical words [N, wpr]: flat uint32 array of
+    kmq_packed_bytes(..., TUNED) / 4 words, padding zero.  Written from the header's formulas, not from the library."""
+    N, wpr = words.shape
+    per = 32 // bits
+    if bits == 4:
+        shifts = [4 * i for i in range(per)]
+    elif bits == 2:
+        shifts = [2 * (i // 4) + 8 * (i % 4) for i in range(per)]
+    else:
+        shifts = [(31 - i // 2) if i % 2 else (15 - i // 2) for i in range(per)]
+    mask = np.uint32((1 << bits) - 1)
+    perm = np.zeros_like(words)
+    for i in range(per):
+        perm |= ((words >> np.uint32(i * bits)) & mask) << np.uint32(shifts[i])
+    steps = -(-wpr // 16)
+    out = np.zeros(-(-N // 16) * steps * 256, dtype=np.uint32)
+    n = np.arange(N)[:, None]
+    j = np.arange(wpr)[None, :]
+    out[(((n // 16) * steps + j // 16) * 16 + n % 16) * 16 + j % 16] = perm
+    return out

@@ -40,8 +40,8 @@ def check_all(idx, cb, x, bits, what=""):
             assert np.array_equal(gu.packed_to_numpy(packed, N), ref_packed), f"{tag}: packed words differ"
         else:
             assert np.array_equal(gu.gpu_unpack(packed, N, K, bits, layout), idx), f"{tag}: unpack(pack(idx)) != idx"
-            pop = int(np.unpackbits(packed.cpu().numpy().view(np.uint8)).sum())
-            assert pop == int(np.unpackbits(ref_packed.view(np.uint8)).sum()), f"{tag}: padding is not zero"
+            assert np.array_equal(packed.cpu().numpy().view(np.uint32), gu.tuned_from_canonical(ref_packed, bits)), \
+                f"{tag}: tuned words differ from the documented layout"
         w = gu.gpu_dequant(packed, cb, N, K, bits, layout)
         assert np.array_equal(w, ref_w), f"{tag}: dequantised weights differ"
         y = gu.gpu_linear(packed, cb, x, N, K, bits, layout)

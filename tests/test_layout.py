@@ -1,0 +1,54 @@
+"""Host-side arithmetic of the two packed layouts (no GPU): the word index map of the tuned layout is injective,
+stays inside kmq_packed_bytes, follows the documented formula, and the field shifts of every bit width are a
+permutation of the canonical ones."""
+import numpy as np
+import pytest
+
+from paper_2602_15563_b200 import build as kb
+from paper_2602_15563_b200 import kmq
+
+C, T = kmq.KMQ_LAYOUT_CANONICAL, kmq.KMQ_LAYOUT_TUNED
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    kb.build()
+
+
+@pytest.mark.parametrize("bits", (1, 2, 4))
+@pytest.mark.parametrize("N,Kwords", [(1, 1), (16, 16), (17, 17), (50, 33), (33, 4)])
+def test_tuned_word_index_is_injective_and_documented(bits, N, Kwords):
+    K = Kwords * (32 // bits)
+    total = kmq.kmq_packed_bytes(N, K, bits, T) // 4
+    steps = -(-Kwords // 16)
+    assert total == -(-N // 16) * steps * 256
+    seen = set()
+    for n in range(N):
+        for j in range(Kwords):
+            w = kmq.kmq_packed_word_index(n, j, N, K, bits, T)
+            assert w == (((n // 16) * steps + j // 16) * 16 + n % 16) * 16 + j % 16
+            assert 0 <= w < total and w not in seen
+            seen.add(w)
+            assert kmq.kmq_packed_word_index(n, j, N, K, bits, C) == n * Kwords + j
+    assert kmq.kmq_packed_word_index(N, 0, N, K, bits, T) == -1
+    assert kmq.kmq_packed_word_index(0, Kwords, N, K, bits, T) == -1
+
+
+@pytest.mark.parametrize("bits", (1, 2, 4))
+def test_field_shifts(bits):
+    per = 32 // bits
+    canon = [kmq.kmq_packed_field_shift(i, bits, C) for i in range(per)]
+    tuned = [kmq.kmq_packed_field_shift(i, bits, T) for i in range(per)]
+    assert canon == [i * bits for i in range(per)]
+    assert sorted(tuned) == canon                                  # same fields, other order
+    covered = np.zeros(32, int)
+    for s in tuned:
+        covered[s:s + bits] += 1
+    assert np.all(covered == 1)                                    # fields tile the word exactly
+    if bits == 4:
+        assert tuned == canon
+    if bits == 2:
+        assert tuned == [2 * (i // 4) + 8 * (i % 4) for i in range(per)]
+    if bits == 1:
+        assert tuned == [(31 - i // 2) if i % 2 else (15 - i // 2) for i in range(per)]
+    assert kmq.kmq_packed_field_shift(per, bits, T) == -1 and kmq.kmq_packed_field_shift(0, 3, T) == -1
