@@ -1,12 +1,12 @@
 // kmq_linear on the tuned (tile-major) layout for batches of 9..64 rows: the decode of a weight fragment is paid
 // once and reused by up to 8 MMAs (one per group of 8 batch rows).
 //
-// One CTA owns 64 output rows = 4 tiles.  Its 8 warps are 2 K-groups of 4 warps; warp (group, i) owns tile i and the
-// steps s = group, group + 2, ... of it.  The 4 warps of a K-group walk the same steps together and share the
-// activations under a step: they are copied global -> shared with cp.async, double buffered, one named barrier per
+// One CTA owns TPC = 4 (or 2) tiles of 16 output rows.  Its 8 warps are 8 / TPC K-groups of TPC warps; warp
+// (group, i) owns tile i and the steps s = group, group + 8 / TPC, ... of it.  The warps of a K-group walk the
+// same steps together and share the activations under a step: they are copied global -> shared with cp.async, double buffered, one named barrier per
 // step.  Per step a warp decodes its 1 KB of packed indices (two 128-bit loads issued one step earlier) into
 // mma.sync.m16n8k16 A fragments and multiplies each fragment with the NT B fragments (batch rows 8 nt .. 8 nt + 7)
-// read from shared memory.  At the end the second K-group hands its accumulators to the first through shared
+// read from shared memory.  At the end the other K-groups hand their accumulators to the first through shared
 // memory, which adds them, applies the b = 1 codebook and stores bf16.
 //
 // b = 4 uses single-entry per-row tables here (16 entries x 32 lane banks, 4 KB per tile; one LDS per weight and a
@@ -21,10 +21,8 @@ namespace {
 
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
-constexpr int kTilesPerCta = 4;
-constexpr int kGroups = 2;
-constexpr int kGroupThreads = 128;
 constexpr int kTableBytesPerTile = 2 * 16 * 32 * 4;   // b = 4: [half][entry][lane] words
+constexpr int kMaxSmem = 200 * 1024;                  // dynamic shared memory a variant may ask for
 
 template <int BITS>
 struct MGeo {
@@ -35,17 +33,19 @@ struct MGeo {
   static constexpr int kChunkStride = kChunkXBytes + 16;  // +16 bytes: conflict-free 16-byte B-fragment loads
   static constexpr int kRowStride = 4 * kChunkStride;     // one batch row of one step
   static constexpr int kPiecesPerRow = kStepK / 8;        // 16-byte pieces per batch row and step
-  static constexpr int kTableBytes = BITS == 4 ? kTilesPerCta * kTableBytesPerTile : 0;
 };
 
-template <int BITS, int NT>
+// TPC tiles per CTA (2 or 4) -> 8 / TPC K-groups of TPC warps
+template <int BITS, int NT, int TPC>
 struct MSmem {
   using G = MGeo<BITS>;
-  static constexpr int kBuf = 8 * NT * G::kRowStride;            // one x buffer: 8 NT batch rows of one step
-  static constexpr int kX = kGroups * 2 * kBuf;                  // double buffered, per K-group
-  static constexpr int kRed = kTilesPerCta * 32 * NT * 4 * 4;    // accumulators of the second K-group (aliases x)
-  static constexpr int kSums = kGroups * 8 * NT * 4;             // b = 1: sum of x per batch row and K-group
-  static constexpr int kTotal = G::kTableBytes + (kX > kRed ? kX : kRed) + kSums;
+  static constexpr int kGroups = kWarps / TPC;
+  static constexpr int kTableBytes = BITS == 4 ? TPC * kTableBytesPerTile : 0;
+  static constexpr int kBuf = 8 * NT * G::kRowStride;                 // one x buffer: 8 NT batch rows of one step
+  static constexpr int kX = kGroups * 2 * kBuf;                       // double buffered, per K-group
+  static constexpr int kRed = (kGroups - 1) * TPC * 32 * NT * 4 * 4;  // accumulators of K-groups 1.. (aliases x)
+  static constexpr int kSums = kGroups * 8 * NT * 4;                  // b = 1: sum of x per batch row and K-group
+  static constexpr int kTotal = kTableBytes + (kX > kRed ? kX : kRed) + kSums;
 };
 
 template <int BITS>
@@ -62,31 +62,33 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src,
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void group_barrier(int group) {
-  asm volatile("bar.sync %0, %1;" ::"r"(group + 1), "r"(kGroupThreads) : "memory");
+__device__ __forceinline__ void group_barrier(int group, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(group + 1), "r"(threads) : "memory");
 }
 
-template <int BITS, int NT>
-__global__ void __launch_bounds__(kThreads, 1) linear_multi_kernel(const uint32_t* __restrict__ packed,
+template <int BITS, int NT, int TPC>
+__global__ void __launch_bounds__(kThreads, (NT <= 2 && TPC == 2) ? 2 : 1) linear_multi_kernel(const uint32_t* __restrict__ packed,
                                                                     const uint16_t* __restrict__ cb,
                                                                     const uint16_t* __restrict__ x,
                                                                     uint16_t* __restrict__ y, int64_t N, int64_t K,
                                                                     int M) {
   using G = MGeo<BITS>;
-  using SM = MSmem<BITS, NT>;
+  using SM = MSmem<BITS, NT, TPC>;
   constexpr int Q = G::kMmaPerWord;
+  constexpr int kGroups = SM::kGroups, kGroupThreads = TPC * 32;
+  constexpr int kSumRows = 8 * NT / TPC;   // b = 1: batch rows whose activations one warp sums
   extern __shared__ __align__(128) unsigned char smem_raw[];
   unsigned char* const tables = smem_raw;
-  unsigned char* const xbase = smem_raw + G::kTableBytes;
+  unsigned char* const xbase = smem_raw + SM::kTableBytes;
   float* const red = reinterpret_cast<float*>(xbase);                       // reused after the main loop
   float* const sums = reinterpret_cast<float*>(xbase + (SM::kX > SM::kRed ? SM::kX : SM::kRed));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int wt = warp & 3, group = warp >> 2;          // tile inside the CTA, K-group
-  const int gtid = threadIdx.x & (kGroupThreads - 1);  // thread inside the K-group
+  const int wt = warp % TPC, group = warp / TPC;       // tile inside the CTA, K-group
+  const int gtid = threadIdx.x - group * kGroupThreads;  // thread inside the K-group
   const int64_t tiles = (N + kTileRows - 1) / kTileRows;
-  const int64_t tile_id = (int64_t)blockIdx.x * kTilesPerCta + wt;
+  const int64_t tile_id = (int64_t)blockIdx.x * TPC + wt;
   const bool has_tile = tile_id < tiles;               // warp-uniform; such a warp still stages x and joins barriers
   const int64_t row0 = tile_id * kTileRows;
   const int chunks = (int)(K / (4 * G::kWordK));
@@ -130,9 +132,9 @@ __global__ void __launch_bounds__(kThreads, 1) linear_multi_kernel(const uint32_
   }
   if constexpr (BITS == 4) {
     // word (tile, half, entry e, lane) = C_row[e] in both halves, row = 16 tile + 8 half + lane / 4
-    for (int i = threadIdx.x; i < kTilesPerCta * 2 * 16 * 32; i += kThreads) {
+    for (int i = threadIdx.x; i < TPC * 2 * 16 * 32; i += kThreads) {
       const int ln = i & 31, e = (i >> 5) & 15, half = (i >> 9) & 1, tl = i >> 10;
-      const int64_t r = min(((int64_t)blockIdx.x * kTilesPerCta + tl) * kTileRows + 8 * half + (ln >> 2), N - 1);
+      const int64_t r = min(((int64_t)blockIdx.x * TPC + tl) * kTileRows + 8 * half + (ln >> 2), N - 1);
       const uint32_t c = __ldg(cb + r * 16 + e);
       reinterpret_cast<uint32_t*>(tables)[i] = c | (c << 16);
     }
@@ -144,10 +146,10 @@ __global__ void __launch_bounds__(kThreads, 1) linear_multi_kernel(const uint32_
   float acc[NT][4];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-  // b = 1: warp wt of a K-group sums the activations of batch rows m = wt, wt + 4, ... (2 NT of them)
-  float sacc[2 * NT];
+  // b = 1: warp wt of a K-group sums the activations of batch rows m = wt, wt + TPC, ...
+  float sacc[kSumRows];
 #pragma unroll
-  for (int i = 0; i < 2 * NT; ++i) sacc[i] = 0.f;
+  for (int i = 0; i < kSumRows; ++i) sacc[i] = 0.f;
 
   for (int s0 = group; s0 < steps; s0 += 2 * kGroups) {   // uniform over the K-group
 #pragma unroll
@@ -155,7 +157,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_multi_kernel(const uint32_
     const int s = s0 + buf * kGroups;
     if (s >= steps) break;
     cp_async_wait_all();
-    group_barrier(group);   // x of step s is in place, and every warp of the group is done with step s - 2
+    group_barrier(group, kGroupThreads);   // x of step s is in place, and every warp of the group is done with step s - 2
     if (s + kGroups < steps) stage(s + kGroups, buf ^ 1);
     const unsigned char* const xs = xgroup + buf * SM::kBuf;
     if (has_tile) {
@@ -214,8 +216,8 @@ __global__ void __launch_bounds__(kThreads, 1) linear_multi_kernel(const uint32_
     if constexpr (BITS == 1) {
       // S[m] = sum_k x[m,k]: the 512 staged activations of a batch row as two 16x16 A tiles times ones
 #pragma unroll
-      for (int i = 0; i < 2 * NT; ++i) {
-        const int m = wt + 4 * i;
+      for (int i = 0; i < kSumRows; ++i) {
+        const int m = wt + TPC * i;
         if (m < M) {
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
@@ -230,22 +232,22 @@ __global__ void __launch_bounds__(kThreads, 1) linear_multi_kernel(const uint32_
    }
   }
 
-  // ---- K-group 1 hands its partial sums to K-group 0, which adds, applies the codebook (b = 1) and stores ----
+  // ---- K-groups 1.. hand their partial sums to K-group 0, which adds, applies the codebook (b = 1) and stores ----
   if constexpr (BITS == 1) {
 #pragma unroll
-    for (int i = 0; i < 2 * NT; ++i) {
+    for (int i = 0; i < kSumRows; ++i) {
       float v = sacc[i];
       v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
       v += __shfl_xor_sync(0xFFFFFFFFu, v, 8);
       v += __shfl_xor_sync(0xFFFFFFFFu, v, 16);
-      if (lane == 0) sums[group * 8 * NT + wt + 4 * i] = v;   // lanes with t = 0 cover every row once
+      if (lane == 0) sums[group * 8 * NT + wt + TPC * i] = v;   // lanes with t = 0 cover every row once
     }
   }
   __syncthreads();   // every warp is done with the x buffers; `red` aliases them
-  if (group == 1) {
+  if (group > 0) {
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
-      *reinterpret_cast<float4*>(red + ((wt * NT + nt) * 32 + lane) * 4) =
+      *reinterpret_cast<float4*>(red + ((((group - 1) * TPC + wt) * NT + nt) * 32 + lane) * 4) =
           make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
   }
   __syncthreads();
@@ -257,8 +259,13 @@ __global__ void __launch_bounds__(kThreads, 1) linear_multi_kernel(const uint32_
     }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      const float4 o = *reinterpret_cast<const float4*>(red + ((wt * NT + nt) * 32 + lane) * 4);
-      const float v[4] = {acc[nt][0] + o.x, acc[nt][1] + o.y, acc[nt][2] + o.z, acc[nt][3] + o.w};
+      float v[4] = {acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]};
+#pragma unroll
+      for (int gq = 1; gq < kGroups; ++gq) {
+        const float4 o =
+            *reinterpret_cast<const float4*>(red + ((((gq - 1) * TPC + wt) * NT + nt) * 32 + lane) * 4);
+        v[0] += o.x; v[1] += o.y; v[2] += o.z; v[3] += o.w;
+      }
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
         const int m = nt * 8 + 2 * t + (r & 1);
@@ -266,7 +273,9 @@ __global__ void __launch_bounds__(kThreads, 1) linear_multi_kernel(const uint32_
         if (m < M && n < N) {
           float out = v[r];
           if constexpr (BITS == 1) {
-            const float sx = sums[m] + sums[8 * NT + m];
+            float sx = 0.f;
+#pragma unroll
+            for (int gq = 0; gq < kGroups; ++gq) sx += sums[gq * 8 * NT + m];
             const uint32_t c = (r >> 1) ? cw1 : cw0;
             const float c0 = bf16_bits_to_float(c & 0xFFFFu), c1 = bf16_bits_to_float(c >> 16);
             out = fmaf(c0, 0.5f * (sx + out), c1 * (0.5f * (sx - out)));
@@ -278,34 +287,50 @@ __global__ void __launch_bounds__(kThreads, 1) linear_multi_kernel(const uint32_
   }
 }
 
-template <int BITS, int NT>
+template <int BITS, int NT, int TPC>
 cudaError_t launch_nt(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N, int64_t K,
                       int M, cudaStream_t s) {
-  constexpr int smem = MSmem<BITS, NT>::kTotal;
+  constexpr int smem = MSmem<BITS, NT, TPC>::kTotal;
   static bool configured[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 64 && !configured[dev]) {
     cudaError_t e =
-        cudaFuncSetAttribute(linear_multi_kernel<BITS, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaFuncSetAttribute(linear_multi_kernel<BITS, NT, TPC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   const int64_t tiles = (N + kTileRows - 1) / kTileRows;
-  const unsigned grid = (unsigned)((tiles + kTilesPerCta - 1) / kTilesPerCta);
-  linear_multi_kernel<BITS, NT><<<grid, kThreads, smem, s>>>(packed, cb, x, y, N, K, M);
+  const unsigned grid = (unsigned)((tiles + TPC - 1) / TPC);
+  linear_multi_kernel<BITS, NT, TPC><<<grid, kThreads, smem, s>>>(packed, cb, x, y, N, K, M);
   return cudaGetLastError();
 }
 
 template <int BITS>
 cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                         int64_t K, int M, cudaStream_t s) {
-  if (M <= 16) return launch_nt<BITS, 2>(packed, cb, x, y, N, K, M, s);
-  if (M <= 32) return launch_nt<BITS, 4>(packed, cb, x, y, N, K, M, s);
+  // Tiles per CTA: 4 share the staged activations among more warps, 2 give twice as many CTAs.  Measured: 2 wins
+  // when 4 would leave more than half of the SMs without a CTA, and for b = 2, 4 at up to 16 rows (two CTAs then fit an SM).
+  const DeviceInfo* di = device_info();
+  const int64_t tiles = (N + kTileRows - 1) / kTileRows;
+  const bool few = (tiles + 3) / 4 <= (di ? di->sm_count : 148) / 2;
+  if (M <= 16) {
+    if (few || BITS != 1) return launch_nt<BITS, 2, 2>(packed, cb, x, y, N, K, M, s);
+    return launch_nt<BITS, 2, 4>(packed, cb, x, y, N, K, M, s);
+  }
+  if (M <= 32) {
+    if constexpr (MSmem<BITS, 4, 2>::kTotal <= kMaxSmem) {
+      if (few) return launch_nt<BITS, 4, 2>(packed, cb, x, y, N, K, M, s);
+    }
+    return launch_nt<BITS, 4, 4>(packed, cb, x, y, N, K, M, s);
+  }
   if constexpr (BITS == 1) {
     return cudaErrorInvalidValue;   // unreachable: b = 1 is launched in passes of at most 32 rows
   } else {
-    return launch_nt<BITS, 8>(packed, cb, x, y, N, K, M, s);
+    if constexpr (MSmem<BITS, 8, 2>::kTotal <= kMaxSmem) {
+      if (few) return launch_nt<BITS, 8, 2>(packed, cb, x, y, N, K, M, s);
+    }
+    return launch_nt<BITS, 8, 4>(packed, cb, x, y, N, K, M, s);
   }
 }
 
