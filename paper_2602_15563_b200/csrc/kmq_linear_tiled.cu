@@ -194,7 +194,10 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
 #pragma unroll
           for (int q2 = 0; q2 < Q; q2 += 2) {
             // 16 bytes of x = the 8 weights of two consecutive MMAs
-            const uint4 xv = *reinterpret_cast<const uint4*>(xb + (j * Q + q2) * 8);
+            // b = 4 is bound by the shared-memory pipe: there only the lanes of real batch rows read (a 128-bit
+            // load takes one pass per quarter warp that has an active lane); elsewhere the predicate costs more
+            uint4 xv = make_uint4(0, 0, 0, 0);
+            if (BITS != 4 || g < M) xv = *reinterpret_cast<const uint4*>(xb + (j * Q + q2) * 8);
 #pragma unroll
             for (int qq = 0; qq < 2; ++qq) {
               const int q = q2 + qq;
