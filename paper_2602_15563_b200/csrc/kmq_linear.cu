@@ -12,7 +12,7 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
     const bool tuned = layout == KMQ_LAYOUT_TUNED;
     p.variant = tuned ? kVariantTiled : kVariantMma;
     p.launches = (int)((M + 7) / 8);
-    if (tuned && M > 8) {
+    if (tuned && M >= linear_multi_min_rows(bits, N)) {
       const int64_t per = linear_multi_rows_per_launch(bits);
       p.variant = kVariantMulti;
       p.launches = (int)((M + per - 1) / per);

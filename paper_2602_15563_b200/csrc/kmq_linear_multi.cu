@@ -1,5 +1,6 @@
-// kmq_linear on the tuned (tile-major) layout for batches of 9..64 rows: the decode of a weight fragment is paid
-// once and reused by up to 8 MMAs (one per group of 8 batch rows).
+// kmq_linear on the tuned (tile-major) layout for batches of up to 64 rows per launch (chosen from 4, 5 or 9 rows
+// on, see linear_multi_min_rows): the tiles of a CTA share the staged activations, and the decode of a weight
+// fragment is paid once and reused by up to 8 MMAs (one per group of 8 batch rows).
 //
 // One CTA owns TPC = 4 (or 2) tiles of 16 output rows.  Its 8 warps are 8 / TPC K-groups of TPC warps; warp
 // (group, i) owns tile i and the steps s = group, group + 8 / TPC, ... of it.  The warps of a K-group walk the
@@ -314,6 +315,10 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
   const DeviceInfo* di = device_info();
   const int64_t tiles = (N + kTileRows - 1) / kTileRows;
   const bool few = (tiles + 3) / 4 <= (di ? di->sm_count : 148) / 2;
+  if (M <= 8) {
+    if (few || BITS != 1) return launch_nt<BITS, 1, 2>(packed, cb, x, y, N, K, M, s);
+    return launch_nt<BITS, 1, 4>(packed, cb, x, y, N, K, M, s);
+  }
   if (M <= 16) {
     if (few || BITS != 1) return launch_nt<BITS, 2, 2>(packed, cb, x, y, N, K, M, s);
     return launch_nt<BITS, 2, 4>(packed, cb, x, y, N, K, M, s);
@@ -339,6 +344,17 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
 // Batch rows per launch of the multi-tile kernel: 64, or 32 for b = 1 (its x buffers are twice as large).
 int linear_multi_rows_per_launch(int bits) { return bits == 1 ? 32 : 64; }
 
+// Smallest batch that goes to the multi-tile kernel.  The GEMV kernel stages the activations of a step once per
+// warp and tile; at b = 1 a step spans 512 activations per batch row against 1 KB of packed words, so from 4 batch
+// rows on sharing the staged activations among the tiles of a CTA wins (8192 x 28672, M = 8: 88 -> 37 us).  At
+// b = 2, 4 it only wins from 5 rows on and when the GEMV grid would not fit the SMs in one wave of CTAs.
+int linear_multi_min_rows(int bits, int64_t N) {
+  if (bits == 1) return 4;
+  const DeviceInfo* di = device_info();
+  const int64_t tiles = (N + kTileRows - 1) / kTileRows;
+  return (di && tiles > (int64_t)di->sm_count * 3) ? 5 : 9;
+}
+
 cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                 int64_t K, int bits, int64_t M, cudaStream_t s) {
   const int64_t per = linear_multi_rows_per_launch(bits);
@@ -347,7 +363,7 @@ cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, cons
     const uint16_t* xp = x + m0 * K;
     uint16_t* yp = y + m0 * N;
     cudaError_t e;
-    if (mc <= 8) e = launch_linear_tiled(packed, cb, xp, yp, N, K, bits, mc, s);   // a short tail
+    if (mc < linear_multi_min_rows(bits, N)) e = launch_linear_tiled(packed, cb, xp, yp, N, K, bits, mc, s);   // a short tail
     else if (bits == 1) e = launch_bits<1>(packed, cb, xp, yp, N, K, mc, s);
     else if (bits == 2) e = launch_bits<2>(packed, cb, xp, yp, N, K, mc, s);
     else e = launch_bits<4>(packed, cb, xp, yp, N, K, mc, s);

@@ -1,4 +1,5 @@
-// kmq_linear on the tuned (tile-major) packed layout, batch rows M <= 8 per pass.
+// kmq_linear on the tuned (tile-major) packed layout, small batches (M <= 8; larger ones and, at b = 1, M >= 4 go
+// to the multi-tile kernel).
 //
 // One CTA owns one tile of 16 output rows; its 8 warps split K step by step (a step = 64 packed bytes of each
 // row = 1 KB of the tile, stored contiguously).  Per step a warp
@@ -419,7 +420,11 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
   if (M == 1) return launch_one<BITS, 1>(packed, cb, x, y, N, K, M, s);
   if (M == 2) return launch_one<BITS, 2>(packed, cb, x, y, N, K, M, s);
   if (M <= 4) return launch_one<BITS, 4>(packed, cb, x, y, N, K, M, s);
-  return launch_one<BITS, 8>(packed, cb, x, y, N, K, M, s);
+  if constexpr (BITS == 1) {
+    return cudaErrorInvalidValue;   // unreachable: b = 1 goes to the multi-tile kernel from 4 batch rows on
+  } else {
+    return launch_one<BITS, 8>(packed, cb, x, y, N, K, M, s);
+  }
 }
 
 template <int BITS, int MMAX>
@@ -448,7 +453,7 @@ cudaError_t launch_split_bits(const uint32_t* packed, const uint16_t* cb, const 
   if (M == 1) return launch_split_one<BITS, 1>(packed, cb, x, y, N, K, M, scratch, ctas, s);
   if (M == 2) return launch_split_one<BITS, 2>(packed, cb, x, y, N, K, M, scratch, ctas, s);
   if (M <= 4) return launch_split_one<BITS, 4>(packed, cb, x, y, N, K, M, scratch, ctas, s);
-  return launch_split_one<BITS, 8>(packed, cb, x, y, N, K, M, scratch, ctas, s);
+  return cudaErrorInvalidValue;   // unreachable: with more tiles than CTA slots, 5 rows and more go to the multi-tile kernel
 }
 
 }  // namespace
@@ -477,11 +482,14 @@ namespace kmq {
 // Every range restarts the load pipeline and the decode set-up once or twice more than a whole tile would, so this
 // only pays when a tile is long: at least kSplitMinSteps steps (measured: 8192 x 28672, b = 4, 224 steps, 55 -> 44 us;
 // with 16..56 steps per tile the per-tile grid is faster).
-constexpr int64_t kSplitMinSteps = 128;
+#ifndef KMQ_SPLIT_MIN_STEPS
+#define KMQ_SPLIT_MIN_STEPS 128
+#endif
+constexpr int64_t kSplitMinSteps = KMQ_SPLIT_MIN_STEPS;
 
 int linear_split_ctas(int64_t N, int64_t K, int bits, int64_t M) {
   const DeviceInfo* di = device_info();
-  if (!di || M > 8) return 0;
+  if (!di || M >= linear_multi_min_rows(bits, N)) return 0;
   const int64_t slots = (int64_t)di->sm_count * 3;
   const int64_t tiles = (N + kRows - 1) / kRows;
   const int64_t steps = (K * bits / 128 + 3) / 4;

@@ -7,8 +7,9 @@ namespace kmq {
 enum LinearVariant : int {
   kVariantGeneric = 0,   // any legal shape and layout, CUDA-core FMAs, one warp per output row
   kVariantMma = 1,       // canonical layout, K*bits % 128 == 0: tensor-core GEMV, activations staged per warp
-  kVariantTiled = 2,     // tuned (tile-major) layout: tensor-core GEMV with coalesced 1 KB steps, M <= 8
-  kVariantMulti = 3,     // tuned layout, M > 8: 64 rows per CTA, one decode feeds up to 8 MMAs
+  kVariantTiled = 2,     // tuned (tile-major) layout: tensor-core GEMV with coalesced 1 KB steps, small batches (M <= 8)
+  kVariantMulti = 3,     // tuned layout, M >= linear_multi_min_rows(): 32 or 64 rows per CTA share the staged
+                         // activations, one decode feeds up to 8 MMAs
   kVariantSplit = 4,     // tuned layout, M <= 8, more tiles than resident CTAs: equal step ranges + fix-up (scratch)
 };
 
@@ -26,6 +27,7 @@ size_t linear_split_scratch_bytes(int ctas);
 cudaError_t launch_linear_split(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                 int64_t K, int bits, int64_t M, void* scratch, int ctas, cudaStream_t s);
 int linear_multi_rows_per_launch(int bits);
+int linear_multi_min_rows(int bits, int64_t N);   // smallest batch routed to the multi-tile kernel
 cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                 int64_t K, int bits, int64_t M, cudaStream_t s);
 

@@ -85,7 +85,7 @@ def test_config4_batch_sweep_8192(M):
     run_case(4, "square8192", 2, M, check_dequant=(M == 1))
 
 
-@pytest.mark.parametrize("M", (1, 16))
+@pytest.mark.parametrize("M", (1, 5, 16))
 @pytest.mark.parametrize("bits", (1, 4))
 def test_config5_large_down_projection(bits, M):
     run_case(5, "down_large", bits, M, check_dequant=(M == 1))
