@@ -170,6 +170,20 @@ kmq_status kmq_linear_static_scratch(const uint32_t* packed, const uint16_t* cod
 size_t kmq_static_scratch_capacity(void);
 
 /*
+ * kmq_device_error_flags -- error word of the kernels on the current device.
+ * The tensor-memory kernel behind kmq_linear for batches of 16 rows and more
+ * (tuned layout) waits on hardware barriers for its asynchronous matrix
+ * instructions; every such wait has an iteration limit, and a CTA whose wait
+ * runs out stops, frees its tensor memory, stores nothing and sets bit 0 here
+ * (the outputs of that call are then incomplete).  The call synchronises the
+ * device, writes the word to *flags (host pointer) and clears it.  0 = no
+ * kernel gave up since the last call.
+ * Errors: KMQ_ERR_NULL, KMQ_ERR_CUDA.
+ */
+#define KMQ_DEVICE_ERROR_WAIT_TIMEOUT 1u
+kmq_status kmq_device_error_flags(unsigned int* flags);
+
+/*
  * kmq_dequant_to_bf16 -- materialise W^[n,k] = C_n[idx[n,k]] as a dense bf16
  * matrix; every element is a bit-exact copy of a stored centroid.  This is
  * the separate dequantise step the paper suggests ahead of a standard GEMM

@@ -2,6 +2,7 @@
 #include <mutex>
 
 #include "kmq_common.cuh"
+#include "kmq_linear_variants.cuh"
 
 namespace kmq {
 
@@ -145,6 +146,11 @@ kmq_status kmq_linear_host(const uint32_t* packed, const uint16_t* codebooks, co
     return s;
   if (cudaMemcpyAsync(y_host, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KMQ_ERR_CUDA;
   return cudaStreamSynchronize(st) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
+}
+
+kmq_status kmq_device_error_flags(unsigned int* flags) {
+  if (!flags) return KMQ_ERR_NULL;
+  return read_device_error_flags(flags) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
 }
 
 kmq_status kmq_dequant_to_bf16(const uint32_t* packed, const uint16_t* codebooks, uint16_t* W, int64_t N, int64_t K,

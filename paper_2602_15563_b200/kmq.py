@@ -39,6 +39,7 @@ SIGNATURES = {
     "kmq_linear_host": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr, _ptr, _ptr, _sz, _ptr]),
     "kmq_linear_static_scratch": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr]),
     "kmq_static_scratch_capacity": (_sz, []),
+    "kmq_device_error_flags": (_int, [_ptr]),
     "kmq_dequant_to_bf16": (_int, [_ptr, _ptr, _ptr, _i64, _i64, _int, _int, _ptr]),
 }
 
@@ -167,6 +168,13 @@ def kmq_linear_static_scratch(packed, codebooks, x, y, N, K, bits, M, layout=KMQ
 
 def kmq_static_scratch_capacity() -> int:
     return lib().kmq_static_scratch_capacity()
+
+
+def kmq_device_error_flags() -> int:
+    """Synchronise the device; return and clear the error word of the kernels (0 = no bounded wait ran out)."""
+    flags = ctypes.c_uint(0)
+    _check(lib().kmq_device_error_flags(ctypes.addressof(flags)), "kmq_device_error_flags")
+    return flags.value
 
 
 def kmq_dequant_to_bf16(packed, codebooks, W, N, K, bits, layout=KMQ_LAYOUT_CANONICAL, stream=None, check=True) -> int:
