@@ -1,25 +1,27 @@
 // kmq_linear on the tuned (tile-major) layout for batches of 16 rows and more: the 5th-generation tensor core
-// (tcgen05.mma, accumulator in tensor memory) multiplies dequantised bf16 weight tiles with the activations.
+// (tcgen05.mma) multiplies dequantised bf16 weights, held in tensor memory, with the activations in shared memory;
+// the accumulator lives in tensor memory too.
 //
-// One CTA owns 128 output rows = 8 tiles of 16; warp w decodes tile w.  K is walked in stages of 128 weights per
-// row.  Per stage
-//   * every lane rebuilds 2 x 32 weights (rows r and r + 8 of its tile, r = lane % 8, 16-byte chunk t = lane / 8
-//     of the step) as bf16 and stores them, 8 weights per 128-bit store, into the A buffer of the stage in the
-//     K-major core-matrix layout the tensor core reads: 8 rows x 16 bytes contiguous, the next 8 weights of the same
-//     rows kLBO bytes further, the next 8 rows kSBO bytes further (a quarter warp fills one core matrix, so the
-//     stores have no bank conflicts);
-//   * the activations under the stage (NB batch rows, zero-filled past M and past K) are copied global -> shared
-//     with cp.async into the B buffer in the same layout;
-//   * after a CTA barrier one thread issues 8 tcgen05.mma (128 x NB x 16 each) that add into the accumulator
-//     D[128 output rows][NB batch rows] in tensor memory, and commits them to the mbarrier of the buffer.
-// Two buffers: the warps decode stage i + 1 while the tensor core works on stage i.  At the end the accumulator is read
-// with tcgen05.ld (lane = output row, column = batch row), rounded to bf16 and stored.
+// One CTA owns 128 output rows (8 tiles of 16) and walks K in stages of 256 (b = 4: 128) weights per row.  Its 8
+// decoder warps and one MMA warp meet only through mbarriers:
+//   * decoder thread (warp w, lane l) owns output row 32 (w % 4) + l of the CTA -- the tensor-memory lane a warp
+//     may write is fixed by its index -- and half w / 4 of the stage's weights of that row.  In the tile-major layout
+//     the 64 bytes of a row in a step are contiguous, so the thread loads its 16 or 32 bytes directly, rebuilds the
+//     64 or 128 weights as bf16 pairs in registers and writes them with tcgen05.st into the A operand of the stage
+//     (lane = row, 32-bit column c = weights 2c, 2c + 1 of the stage).  The decoder threads also copy the
+//     activations two stages ahead (NB batch rows, zero-filled past M and past K) global -> shared with cp.async
+//     into the K-major core-matrix layout of the B operand (8 rows x 16 bytes contiguous, the next 8 weights kLBO
+//     bytes further, the next 8 rows kSBO bytes further).  When a warp's part of a stage is in place it arrives on
+//     the stage's `full` barrier;
+//   * the MMA warp waits for `full`, issues one tcgen05.mma (128 x NB x 16) per 16 weights that adds into the
+//     accumulator D[128 output rows][NB batch rows], and commits them to the stage's `empty` barrier, which the
+//     decoders wait for before they overwrite the A operand (ring of 2) and the B buffer (ring of 4).
+// At the end the decoder warps read the accumulator with tcgen05.ld (lane = output row, column = batch row), round
+// to bf16 and store.
 //
-// Inside a stage the order of the weights of a row is (chunk t, then the 32 weights of this stage in the chunk);
-// A and B use the same order, and a sum does not depend on the order of its terms.
-//
-// Every wait on an mbarrier is bounded; when it runs out the CTA stops, sets bit 0 of the device error word, frees its
-// tensor memory and returns.
+// Every wait on an mbarrier is bounded; a warp whose wait runs out sets bit 0 of the device error word and goes to
+// the end of the kernel (so does, after its own bounded waits, every warp that depended on it), where the tensor
+// memory is freed.
 #include "kmq_common.cuh"
 #include "kmq_linear_variants.cuh"
 #include "kmq_mma_common.cuh"
@@ -30,55 +32,69 @@ __device__ unsigned int g_device_error_flags = 0;   // sticky; read and cleared 
 
 namespace {
 
-constexpr int kBlockRows = 128;                          // rows of the MMA (UMMA M)
-constexpr int kStageK = 128;                             // weights of a row per stage
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
+constexpr int kBM = 128;                                 // output rows per CTA (rows of the MMA)
+constexpr int kDecodeWarps = 8;
+constexpr int kDecodeThreads = kDecodeWarps * 32;
+constexpr int kThreads = kDecodeThreads + 32;            // + the MMA warp
+constexpr int kARing = 2;                                // A operands in tensor memory
+constexpr int kBRing = 4;                                // B buffers in shared memory (activations run 2 stages ahead)
+#ifndef KMQ_UMMA_WRING
+#define KMQ_UMMA_WRING 8
+#endif
+constexpr int kWRing = KMQ_UMMA_WRING;                   // stages of packed words in flight per thread (cp.async ring)
 constexpr int kLBO = 128;                                // bytes between core matrices that are neighbours in K
-constexpr int kSBO = (kStageK / 8) * kLBO;               // bytes between groups of 8 rows
-constexpr int kAStageBytes = kBlockRows * kStageK * 2;   // 32 KB
-constexpr int kKSlices = kStageK / 16;                   // MMAs per stage
 constexpr uint32_t kWaitLimit = 1u << 20;                // polls of an mbarrier (about 20 ns apart) before giving up
 
 template <int BITS>
 struct UGeo {
-  static constexpr int kWordK = 32 / BITS;
-  static constexpr int kStepK = 512 / BITS;                    // weights of a row per 1 KB step of a tile
-  static constexpr int kChunkK = kStepK / 4;                   // weights under one 16-byte chunk
-  static constexpr int kStagesPerStep = kStepK / kStageK;      // 1, 2, 4 for b = 4, 2, 1
-  static constexpr int kTableBytes = BITS == 4 ? kWarps * 2 * 16 * 128 : 0;   // b = 4: [tile][half][entry][lane]
+  static constexpr int kStageK = BITS == 4 ? 128 : 256;          // weights of a row per stage
+  static constexpr int kStagesPerStep = (512 / BITS) / kStageK;  // 1, 1, 2 for b = 4, 2, 1
+  static constexpr int kThreadBytes = kStageK * BITS / 16;       // packed bytes a thread decodes per stage: 32, 32, 16
+  static constexpr int kCols = kStageK / 2;                      // 32-bit columns of the A operand of a stage
+  static constexpr int kKSlices = kStageK / 16;                  // MMAs per stage
+  static constexpr int kSBO = (kStageK / 8) * kLBO;              // bytes between groups of 8 batch rows in a B buffer
+  static constexpr int kTmemCols = BITS == 4 ? 256 : 512;        // kARing * kCols + up to 64 columns of D, a power of two
+  static constexpr int kTableBytes = BITS == 4 ? 4 * 16 * 128 : 0;   // b = 4: [lane quarter][entry][lane]
 };
 
 template <int BITS, int NB>
 struct USmem {
-  static constexpr int kBStageBytes = NB * kStageK * 2;
-  static constexpr int kA = 0;
-  static constexpr int kB = 2 * kAStageBytes;
-  static constexpr int kTables = kB + 2 * kBStageBytes;
-  static constexpr int kBars = kTables + UGeo<BITS>::kTableBytes;   // two mbarriers, then the tensor-memory address
-  static constexpr int kTotal = kBars + 32;
+  static constexpr int kBStageBytes = NB * UGeo<BITS>::kStageK * 2;
+  static constexpr int kB = 0;
+  static constexpr int kWords = kB + kBRing * kBStageBytes;   // ring of packed words: [stage][16-byte piece][thread]
+  static constexpr int kTables = kWords + kWRing * kDecodeThreads * UGeo<BITS>::kThreadBytes;
+  static constexpr int kBars = kTables + UGeo<BITS>::kTableBytes;   // full[kARing], empty[kARing]
+  static constexpr int kTmemSlot = kBars + 2 * kARing * 8;
+  static constexpr int kTotal = kTmemSlot + 16;
 };
 
 // Shared-memory matrix descriptor: K-major, no swizzle, strides kLBO / kSBO, descriptor version of sm_100.
+template <int SBO>
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(kLBO >> 4) << 16) | ((uint64_t)(kSBO >> 4) << 32) |
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(kLBO >> 4) << 16) | ((uint64_t)(SBO >> 4) << 32) |
          ((uint64_t)1 << 46);
 }
 
-// Instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = NB.
+// Instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, M = kBM, N = NB.
 template <int NB>
 __device__ __forceinline__ uint32_t instr_desc() {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NB >> 3) << 17) | ((uint32_t)(kBlockRows >> 4) << 24);
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NB >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 }
 
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+// D (tensor memory) (+)= A (tensor memory) x B (shared memory descriptor)
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       :
-      : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
+}
+__device__ __forceinline__ void tmem_store8(uint32_t taddr, const uint32_t (&v)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(v[0]),
+               "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -91,8 +107,11 @@ __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_s
   const int bytes = valid ? 16 : 0;   // 0 source bytes: the 16 destination bytes are zero-filled
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gmem_src), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all() {
-  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 // Bounded wait for the phase of parity `parity` of an mbarrier.
@@ -110,7 +129,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   return false;
 }
 
-// Per-row decode state of a lane: rows r (h = 0) and r + 8 (h = 1) of its tile.
+// Decode state of a thread's output row.
 template <int BITS>
 struct RowState;
 template <>
@@ -129,56 +148,54 @@ struct RowState<1> {
 };
 template <>
 struct RowState<4> {
-  const unsigned char* tab;   // this lane's bank of the [entry][lane] table of its tile half
-  __device__ __forceinline__ void init(const uint16_t*, const unsigned char* table_half, int lane) {
-    tab = table_half + lane * 4;
+  const unsigned char* tab;   // this lane's bank of the [entry][lane] table of its lane quarter
+  __device__ __forceinline__ void init(const uint16_t*, const unsigned char* table_quarter, int lane) {
+    tab = table_quarter + lane * 4;
   }
 };
 
-// The 32 weights of stage U (of its step) in one lane's chunk `v` of one row -> four 128-bit stores of 8 bf16 each,
-// kLBO bytes apart.
-template <int BITS, int U>
-__device__ __forceinline__ void decode_store(const uint4& v, const RowState<BITS>& st, unsigned char* dst) {
-  const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
-  if constexpr (BITS == 4) {
+// One packed word of a row -> bf16 pairs in the order of k, written to consecutive columns of the row's
+// tensor-memory lane starting at `taddr`.  Returns the number of columns written (weights per word / 2).
+template <int BITS>
+__device__ __forceinline__ void decode_word_to_tmem(uint32_t w, const RowState<BITS>& st, uint32_t taddr) {
+  if constexpr (BITS == 2) {
+    uint32_t a[8];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t e[8];
+    for (int q = 0; q < 4; ++q) st.d.pair(w, q, a[2 * q], a[2 * q + 1]);   // weights 4q .. 4q + 3
+    tmem_store8(taddr, a);
+  } else if constexpr (BITS == 1) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {   // nibble i -> byte offset nibble * 128 of the lane's table bank
-        const int sh = 4 * i - 7;
-        const uint32_t u = sh < 0 ? (w4[j] << -sh) : (w4[j] >> sh);
-        e[i] = *reinterpret_cast<const uint32_t*>(st.tab + (u & 0x780u));
-      }
-      *reinterpret_cast<uint4*>(dst + j * kLBO) = make_uint4(prmt(e[0], e[1], 0x7610u), prmt(e[2], e[3], 0x7610u),
-                                                             prmt(e[4], e[5], 0x7610u), prmt(e[6], e[7], 0x7610u));
-    }
-  } else if constexpr (BITS == 2) {
-#pragma unroll
-    for (int jj = 0; jj < 2; ++jj) {
-      const uint32_t w = w4[2 * U + jj];
+    for (int h = 0; h < 2; ++h) {
       uint32_t a[8];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) st.d.pair(w, q, a[2 * q], a[2 * q + 1]);   // weights 4q .. 4q + 3
-      *reinterpret_cast<uint4*>(dst + (2 * jj) * kLBO) = make_uint4(a[0], a[1], a[2], a[3]);
-      *reinterpret_cast<uint4*>(dst + (2 * jj + 1) * kLBO) = make_uint4(a[4], a[5], a[6], a[7]);
-    }
-  } else {
-    const uint32_t w = w4[U];
-#pragma unroll
-    for (int kg = 0; kg < 4; ++kg) {
-      uint32_t a[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < 8; ++i) {
         // shift c puts weights (2c, 2c + 1) on bits 15 and 31; PRMT in sign-replicate mode turns them into
-        // 16-bit masks; masked XOR picks c0 or c1 bit-exactly
-        const uint32_t sh = w * kPow2[4 * kg + i];
+        // 16-bit masks; the masked XOR picks c0 or c1 bit-exactly
+        const uint32_t sh = w * kPow2[8 * h + i];
         const uint32_t sel = prmt(sh, sh, 0xBB99u);
         asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(a[i]) : "r"(sel), "r"(st.diff), "r"(st.base));
       }
-      *reinterpret_cast<uint4*>(dst + kg * kLBO) = make_uint4(a[0], a[1], a[2], a[3]);
+      tmem_store8(taddr + 8 * h, a);
     }
   }
+}
+// b = 4: two words (16 weights) per 8 columns
+__device__ __forceinline__ void decode_words4_to_tmem(uint32_t w0, uint32_t w1, const RowState<4>& st, uint32_t taddr) {
+  uint32_t a[8];
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const uint32_t w = j ? w1 : w0;
+    uint32_t e[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {   // nibble i -> byte offset nibble * 128 of the lane's table bank
+      const int sh = 4 * i - 7;
+      const uint32_t u = sh < 0 ? (w << -sh) : (w >> sh);
+      e[i] = *reinterpret_cast<const uint32_t*>(st.tab + (u & 0x780u));
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) a[4 * j + i] = prmt(e[2 * i], e[2 * i + 1], 0x7610u);
+  }
+  tmem_store8(taddr, a);
 }
 
 template <int BITS, int NB>
@@ -190,147 +207,190 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
   using G = UGeo<BITS>;
   using SM = USmem<BITS, NB>;
   constexpr int SPS = G::kStagesPerStep;
-  constexpr uint32_t kTmemCols = NB <= 32 ? 32 : 64;   // a power of two >= 32
+  constexpr int NV = G::kThreadBytes / 16;   // 128-bit loads per thread and stage
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  unsigned char* const a_buf = smem_raw + SM::kA;
   unsigned char* const tables = smem_raw + SM::kTables;
   const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem_raw);
-  const uint32_t a_addr = smem_base + SM::kA, b_addr = smem_base + SM::kB, bar_addr = smem_base + SM::kBars;
-  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + SM::kBars + 16);
+  const uint32_t b_addr = smem_base + SM::kB;
+  const uint32_t full_bar = smem_base + SM::kBars, empty_bar = full_bar + 8 * kARing;
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + SM::kTmemSlot);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r = lane & 7, t = lane >> 3;
-  const int64_t tiles = (N + kTileRows - 1) / kTileRows;
-  const int64_t tile_id = (int64_t)blockIdx.x * kWarps + warp;
-  const bool has_tile = tile_id < tiles;   // warp-uniform; a warp without a tile leaves its A rows as they are
-  const int64_t row0 = tile_id * kTileRows;
-  const int chunks = (int)(K / (4 * G::kWordK));
-  const int steps = (chunks + 3) >> 2;
-  // step s of the tile: 64 16-byte units, unit h * 32 + row * 4 + chunk holds chunk `chunk` of row (row + 8h)
-  const uint4* __restrict__ tile =
-      reinterpret_cast<const uint4*>(packed) + (has_tile ? tile_id : 0) * (int64_t)steps * 64 + r * 4 + t;
+  const int64_t block_row0 = (int64_t)blockIdx.x * kBM;
+  const int chunks = (int)(K / (128 / BITS));   // 16-byte chunks per row
+  const int steps = (chunks + 3) >> 2;          // the layout pads every row to whole steps of 64 bytes
+  const int total = steps * SPS;                // stages
 
-  // ---- set-up: mbarriers, tensor memory, decode state ----
+  // ---- set-up: mbarriers, tensor memory, tables ----
   if (threadIdx.x == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_addr) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_addr + 8) : "memory");
+#pragma unroll
+    for (int i = 0; i < kARing; ++i) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full_bar + 8 * i), "r"(kDecodeWarps) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(empty_bar + 8 * i) : "memory");
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bar_addr + 16), "r"(kTmemCols)
+  if (warp == kDecodeWarps) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_base + SM::kTmemSlot),
+                 "r"((uint32_t)G::kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   if constexpr (BITS == 4) {
-    // word [tile][half][entry e][lane] = (C_row[e], C_row[e]), row = 16 tile + 8 half + lane % 8
-    for (int i = threadIdx.x; i < kWarps * 2 * 16 * 32; i += kThreads) {
-      const int ln = i & 31, e = (i >> 5) & 15, half = (i >> 9) & 1, tl = i >> 10;
-      const int64_t row = min(((int64_t)blockIdx.x * kWarps + tl) * kTileRows + 8 * half + (ln & 7), N - 1);
+    // word [lane quarter q][entry e][lane] = (C_row[e], C_row[e]), row = block_row0 + 32 q + lane
+    for (int i = threadIdx.x; i < 4 * 16 * 32; i += kThreads) {
+      const int ln = i & 31, e = (i >> 5) & 15, q = i >> 9;
+      const int64_t row = min(block_row0 + 32 * q + ln, N - 1);
       const uint32_t c = __ldg(cb + row * 16 + e);
       reinterpret_cast<uint32_t*>(tables)[i] = c | (c << 16);
     }
   }
-  RowState<BITS> st0, st1;
-  st0.init(cb + min(row0 + r, N - 1) * (1 << BITS), tables + (warp * 2 + 0) * 2048, lane);
-  st1.init(cb + min(row0 + r + 8, N - 1) * (1 << BITS), tables + (warp * 2 + 1) * 2048, lane);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem_d = *tmem_slot;
-
-  // this lane's 16-byte slots in an A buffer: row group 2 warp + h, core matrices 4t .. 4t + 3, row r
-  unsigned char* const a_lane = a_buf + (2 * warp) * kSBO + (4 * t) * kLBO + r * 16;
-  const uint32_t idesc = instr_desc<NB>();
-
-  uint4 na = make_uint4(0, 0, 0, 0), nb = na;
-  if (has_tile && steps > 0) {
-    na = ldg_stream_u4(tile);
-    nb = ldg_stream_u4(tile + 32);
-  }
-  int stage = 0;
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_d = tmem_base + kARing * G::kCols;   // the accumulator follows the A operands
   bool ok = true;
-  for (int s = 0; s < steps && ok; ++s) {
-    const uint4 va = na, vb = nb;
-    if (has_tile && s + 1 < steps) {
-      na = ldg_stream_u4(tile + (int64_t)(s + 1) * 64);
-      nb = ldg_stream_u4(tile + (int64_t)(s + 1) * 64 + 32);
-    }
+
+  if (warp < kDecodeWarps) {
+    // ================= decoder warps =================
+    const int q = warp & 3, kh = warp >> 2;   // tensor-memory lane quarter; which half of a stage's weights
+    const int rho = 32 * q + lane;            // output row inside the CTA = tensor-memory lane
+    const int64_t tiles = (N + kTileRows - 1) / kTileRows;
+    const int64_t tile_id = (int64_t)blockIdx.x * (kBM / 16) + (rho >> 4);
+    const bool has_tile = tile_id < tiles;    // rows of a missing tile decode zeros; they are never stored
+    // row rho % 16 of a tile owns bytes [64 (rho % 16), +64) of each 1 KB step
+    const unsigned char* __restrict__ row_bytes = reinterpret_cast<const unsigned char*>(packed) +
+                                                  (has_tile ? tile_id : 0) * (int64_t)steps * 1024 + (rho & 15) * 64;
+    RowState<BITS> st;
+    st.init(cb + min(block_row0 + rho, N - 1) * (1 << BITS), tables + q * 2048, lane);
+    // packed words of stage i: global -> this thread's slot of ring stage i % kWRing (read back by the same thread)
+    unsigned char* const w_slot = smem_raw + SM::kWords + threadIdx.x * 16;   // piece j: kDecodeThreads * 16 bytes further
+    const uint32_t w_slot_addr = smem_base + SM::kWords + threadIdx.x * 16;
+    constexpr int kWStage = kDecodeThreads * G::kThreadBytes;
+    auto copy_words = [&](int i) {
+      const int s = i / SPS, u = i % SPS;
+      const unsigned char* src = row_bytes + (int64_t)s * 1024 + (BITS == 1 ? 32 * u + 16 * kh : 32 * kh);
 #pragma unroll
-    for (int u = 0; u < SPS; ++u) {
-      if (!ok) break;
-      const int buf = stage & 1;
-      if (stage >= 2) {   // the MMAs that read this buffer two stages ago are done
-        ok = mbar_wait(bar_addr + 8 * buf, ((stage >> 1) - 1) & 1);
-        ok = __syncthreads_and(ok);
-        if (!ok) break;
-      }
-      // activations: piece p = (batch row m, core matrix kg); bits of p: kg0 | m0..2 | kg1..3 | m3..
+      for (int j = 0; j < NV; ++j) cp_async16(w_slot_addr + (i % kWRing) * kWStage + j * (kDecodeThreads * 16), src + 16 * j, has_tile);
+    };
+    // activations of stage i -> B buffer i % kBRing; piece p = (batch row m, core matrix kg), bits of p:
+    // kg0 | m0..2 | kg1.. | m3..  (8 consecutive threads: 4 rows x 32 contiguous bytes)
+    auto stage_x = [&](int i) {
+      constexpr int KGS = G::kStageK / 8;
+      const uint32_t dst = b_addr + (i % kBRing) * SM::kBStageBytes;
 #pragma unroll
-      for (int i = 0; i < NB / 16; ++i) {
-        const int p = threadIdx.x + kThreads * i;
-        const int kg = (p & 1) | ((p >> 3) & 14), m = ((p >> 1) & 7) | ((p >> 7) << 3);
-        const int64_t k = (int64_t)s * G::kStepK + (kg >> 2) * G::kChunkK + u * 32 + (kg & 3) * 8;
+      for (int j = 0; j < NB * KGS / kDecodeThreads; ++j) {
+        const int p = threadIdx.x + kDecodeThreads * j;
+        const int kg = (p & 1) | (((p >> 4) & (KGS / 2 - 1)) << 1);
+        const int m = ((p >> 1) & 7) | ((p / (8 * KGS)) << 3);
+        const int64_t k = (int64_t)i * G::kStageK + kg * 8;
         const bool valid = m < M && k < K;
-        cp_async16(b_addr + buf * SM::kBStageBytes + (m >> 3) * kSBO + kg * kLBO + (m & 7) * 16,
-                   x + (valid ? (int64_t)m * K + k : 0), valid);
+        cp_async16(dst + (m >> 3) * G::kSBO + kg * kLBO + (m & 7) * 16, x + (valid ? (int64_t)m * K + k : 0), valid);
       }
-      if (has_tile) {
-        unsigned char* const dst = a_lane + buf * kAStageBytes;
-        if (u == 0) { decode_store<BITS, 0>(va, st0, dst); decode_store<BITS, 0>(vb, st1, dst + kSBO); }
-        if (SPS > 1 && u == 1) { decode_store<BITS, 1 % SPS>(va, st0, dst); decode_store<BITS, 1 % SPS>(vb, st1, dst + kSBO); }
-        if (SPS > 2 && u == 2) { decode_store<BITS, 2 % SPS>(va, st0, dst); decode_store<BITS, 2 % SPS>(vb, st1, dst + kSBO); }
-        if (SPS > 2 && u == 3) { decode_store<BITS, 3 % SPS>(va, st0, dst); decode_store<BITS, 3 % SPS>(vb, st1, dst + kSBO); }
-      }
-      cp_async_wait_all();
-      async_proxy_fence();   // the stores above become visible to the tensor core's reads of shared memory
-      __syncthreads();
-      if (threadIdx.x == 0) {
+      cp_async_commit();
+    };
+
+    // prologue: kWRing groups; group d holds the words of stage d and, for d < 2, the activations of stage d
+#pragma unroll 1
+    for (int d = 0; d < kWRing; ++d) {
+      if (d < total) copy_words(d);
+      if (d < 2 && d < total) stage_x(d);
+      else cp_async_commit();
+    }
+    for (int i = 0; i < total; ++i) {
+      const int abuf = i & 1;
+      cp_async_wait<kWRing - 1>();   // the group of the words of stage i has landed
+      uint4 v[NV];
+#pragma unroll
+      for (int j = 0; j < NV; ++j) v[j] = *reinterpret_cast<const uint4*>(w_slot + (i % kWRing) * kWStage + j * (kDecodeThreads * 16));
+      if (i >= kARing) {
+        // the MMAs of stage i - 2 are done: A operand i % 2 and B buffer (i + 2) % 4 may be overwritten
+        ok = mbar_wait(empty_bar + 8 * abuf, ((i >> 1) - 1) & 1);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
         tc_fence_after_sync();
-#pragma unroll
-        for (int ks = 0; ks < kKSlices; ++ks)
-          umma_bf16(tmem_d, smem_desc(a_addr + buf * kAStageBytes + ks * 2 * kLBO),
-                    smem_desc(b_addr + buf * SM::kBStageBytes + ks * 2 * kLBO), idesc, (stage | ks) != 0);
-        umma_commit(bar_addr + 8 * buf);
       }
-      ++stage;
-    }
-  }
-  // ---- all MMAs done -> read the accumulator, round, store ----
-  if (ok && stage > 0) {
-    const int last = stage - 1;
-    ok = mbar_wait(bar_addr + 8 * (last & 1), (last >> 1) & 1);
-    ok = __syncthreads_and(ok);
-  }
-  if (ok) {
-    tc_fence_after_sync();
-    const int q = warp & 3, half = warp >> 2;   // a warp reads the 32 lanes of its quarter; the two halves split the columns
-    const int64_t n = (int64_t)blockIdx.x * kBlockRows + q * 32 + lane;
+      // this thread's half of the stage's weights of its row -> columns kh * kCols / 2 ... of the A operand
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + abuf * G::kCols + kh * (G::kCols / 2);
 #pragma unroll
-    for (int c0 = 0; c0 < NB / 2; c0 += 8) {
-      const int col = half * (NB / 2) + c0;
-      uint32_t v[8];
-      if (stage > 0) {
-        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-                     : "r"(tmem_d + ((uint32_t)(q * 32) << 16) + col));
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      } else {
+      for (int j = 0; j < NV; ++j) {
+        const uint32_t w4[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+        if constexpr (BITS == 4) {
+          decode_words4_to_tmem(w4[0], w4[1], st, taddr + j * 16);
+          decode_words4_to_tmem(w4[2], w4[3], st, taddr + j * 16 + 8);
+        } else {
+          constexpr int kColsPerWord = 16 / BITS;   // 8 or 16
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = 0;
+          for (int jj = 0; jj < 4; ++jj) decode_word_to_tmem<BITS>(w4[jj], st, taddr + (4 * j + jj) * kColsPerWord);
+        }
       }
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        if (col + j < M && n < N) y[(int64_t)(col + j) * N + n] = (uint16_t)float_to_bf16_bits(__uint_as_float(v[j]));
+      // one group per iteration: the activations of stage i + 2 and the words of stage i + kWRing (its ring slot
+      // was read above, and the decode has consumed what was read)
+      if (i + kWRing < total) copy_words(i + kWRing);
+      if (i + 2 < total) stage_x(i + 2);
+      else cp_async_commit();
+      cp_async_wait<2>();   // the group with the activations of stage i has landed
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      async_proxy_fence();   // the copies into shared memory become visible to the tensor core's reads
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full_bar + 8 * abuf);
     }
-  } else if (threadIdx.x == 0) {
-    atomicOr(&g_device_error_flags, 1u);
+    // ---- all MMAs done -> read the accumulator, round, store ----
+    if (ok && total > 0) {
+      const int last = total - 1;
+      ok = mbar_wait(empty_bar + 8 * (last & 1), (last >> 1) & 1);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+    }
+    if (ok) {
+      tc_fence_after_sync();
+      const int64_t n = block_row0 + rho;
+#pragma unroll
+      for (int c0 = 0; c0 < NB / 2; c0 += 8) {
+        const int col = kh * (NB / 2) + c0;   // the two warps of a lane quarter split the columns
+        uint32_t w[8];
+        if (total > 0) {
+          asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                       : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                       : "r"(tmem_d + ((uint32_t)(q * 32) << 16) + col));
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) w[j] = 0;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (col + j < M && n < N) y[(int64_t)(col + j) * N + n] = (uint16_t)float_to_bf16_bits(__uint_as_float(w[j]));
+      }
+    } else if (lane == 0) {
+      atomicOr(&g_device_error_flags, 1u);
+    }
+  } else if (lane == 0) {
+    // ================= MMA warp (one thread) =================
+    const uint32_t idesc = instr_desc<NB>();
+    for (int i = 0; i < total; ++i) {
+      const int abuf = i & 1;
+      if (!mbar_wait(full_bar + 8 * abuf, (i >> 1) & 1)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after_sync();
+      const uint32_t b_stage = b_addr + (i % kBRing) * SM::kBStageBytes;
+#pragma unroll
+      for (int ks = 0; ks < G::kKSlices; ++ks)
+        umma_bf16(tmem_d, tmem_base + abuf * G::kCols + ks * 8, smem_desc<G::kSBO>(b_stage + ks * 2 * kLBO), idesc,
+                  (i | ks) != 0);
+      umma_commit(empty_bar + 8 * abuf);
+    }
+    if (!ok) atomicOr(&g_device_error_flags, 1u);
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(kTmemCols) : "memory");
+  if (warp == kDecodeWarps)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)G::kTmemCols)
+                 : "memory");
 }
-
 
 }  // namespace
 
@@ -348,7 +408,7 @@ cudaError_t launch_nb(const uint32_t* packed, const uint16_t* cb, const uint16_t
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  const unsigned grid = (unsigned)((N + kBlockRows - 1) / kBlockRows);
+  const unsigned grid = (unsigned)((N + kBM - 1) / kBM);
   linear_umma_kernel<BITS, NB><<<grid, kThreads, smem, s>>>(packed, cb, x, y, N, K, M);
   return cudaGetLastError();
 }
@@ -365,7 +425,7 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
 }  // namespace
 
 #ifndef KMQ_UMMA_MIN_ROWS
-#define KMQ_UMMA_MIN_ROWS (1 << 30)   // not selected yet: correct, but slower than the multi-tile kernel
+#define KMQ_UMMA_MIN_ROWS (1 << 30)
 #endif
 int linear_umma_min_rows() { return KMQ_UMMA_MIN_ROWS; }
 int linear_umma_rows_per_launch() { return 64; }
