@@ -170,11 +170,32 @@ kmq_status kmq_linear_static_scratch(const uint32_t* packed, const uint16_t* cod
 size_t kmq_static_scratch_capacity(void);
 
 /*
+ * kmq_linear_tcgen05 -- the same layer (same operands, result and tolerance
+ * as kmq_linear) computed by the 5th-generation tensor-core path: weights of
+ * 128 output rows are dequantised straight into tensor memory as the A
+ * operand of tcgen05.mma, the activations are the B operand in shared
+ * memory, the accumulator lives in tensor memory.  `packed` must be in
+ * KMQ_LAYOUT_TUNED and K * bits a multiple of 128; any M >= 1 (64 batch rows
+ * per launch).  This is the large-batch design the paper's roofline model
+ * points to (Appendix "Theoretical model": beyond a batch of P_w * nu / 16
+ * the layer is compute bound).  kmq_linear does not select it: one
+ * tcgen05.mma costs at least 69 clocks whatever its N, which caps this design
+ * at about 30 weights per clock and SM, and on B200 the mma.sync kernels are
+ * faster up to the 64 batch rows measured (figures in the design notes).
+ * It needs no workspace.  Its waits on hardware barriers are bounded, see
+ * kmq_device_error_flags.
+ * Errors: KMQ_ERR_NULL, KMQ_ERR_BITS, KMQ_ERR_SHAPE, KMQ_ERR_ALIGN,
+ * KMQ_ERR_CUDA.
+ */
+kmq_status kmq_linear_tcgen05(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x,
+                              uint16_t* y, int64_t N, int64_t K, int bits, int64_t M, void* stream);
+
+/*
  * kmq_device_error_flags -- error word of the kernels on the current device.
- * The tensor-memory kernel behind kmq_linear for batches of 16 rows and more
- * (tuned layout) waits on hardware barriers for its asynchronous matrix
- * instructions; every such wait has an iteration limit, and a CTA whose wait
- * runs out stops, frees its tensor memory, stores nothing and sets bit 0 here
+ * The tensor-memory kernel behind kmq_linear_tcgen05 waits on hardware
+ * barriers for its asynchronous matrix instructions; every such wait has an
+ * iteration limit, and a warp whose wait runs out stops, stores nothing and
+ * sets bit 0 here; the CTA still frees its tensor memory
  * (the outputs of that call are then incomplete).  The call synchronises the
  * device, writes the word to *flags (host pointer) and clears it.  0 = no
  * kernel gave up since the last call.

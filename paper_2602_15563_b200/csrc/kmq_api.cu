@@ -148,6 +148,17 @@ kmq_status kmq_linear_host(const uint32_t* packed, const uint16_t* codebooks, co
   return cudaStreamSynchronize(st) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
 }
 
+kmq_status kmq_linear_tcgen05(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x, uint16_t* y,
+                              int64_t N, int64_t K, int bits, int64_t M, void* stream) {
+  if (!packed || !codebooks || !x || !y) return KMQ_ERR_NULL;
+  if (kmq_status s = check_shape(N, K, bits, M)) return s;
+  if ((K * bits) % 128 != 0) return KMQ_ERR_SHAPE;
+  if (!aligned16(packed) || !aligned16(codebooks) || !aligned16(x) || !aligned16(y)) return KMQ_ERR_ALIGN;
+  if (!device_info()) return KMQ_ERR_CUDA;
+  return launch_linear_umma(packed, codebooks, x, y, N, K, bits, M, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK
+                                                                                                        : KMQ_ERR_CUDA;
+}
+
 kmq_status kmq_device_error_flags(unsigned int* flags) {
   if (!flags) return KMQ_ERR_NULL;
   return read_device_error_flags(flags) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;

@@ -12,13 +12,6 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
     const bool tuned = layout == KMQ_LAYOUT_TUNED;
     p.variant = tuned ? kVariantTiled : kVariantMma;
     p.launches = (int)((M + 7) / 8);
-    if (tuned && M >= linear_umma_min_rows()) {
-      const int64_t per = linear_umma_rows_per_launch();
-      p.variant = kVariantUmma;
-      p.launches = (int)((M + per - 1) / per);
-      p.name = bits == 4 ? "umma_table_b4" : bits == 2 ? "umma_prmt_b2" : "umma_select_b1";
-      return p;
-    }
     if (tuned && M >= linear_multi_min_rows(bits, N)) {
       const int64_t per = linear_multi_rows_per_launch(bits);
       p.variant = kVariantMulti;
@@ -54,8 +47,6 @@ cudaError_t launch_linear(const LinearPlan& plan, const uint32_t* packed, const 
   switch (plan.variant) {
     case kVariantSplit:
       return launch_linear_split(packed, cb, x, y, N, K, bits, M, workspace, plan.split_k, s);
-    case kVariantUmma:
-      return launch_linear_umma(packed, cb, x, y, N, K, bits, M, s);
     case kVariantMulti:
       return launch_linear_multi(packed, cb, x, y, N, K, bits, M, s);
     case kVariantTiled:

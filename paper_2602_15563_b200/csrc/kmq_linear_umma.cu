@@ -33,27 +33,31 @@ __device__ unsigned int g_device_error_flags = 0;   // sticky; read and cleared 
 namespace {
 
 constexpr int kBM = 128;                                 // output rows per CTA (rows of the MMA)
-constexpr int kDecodeWarps = 8;
+constexpr int kDecodeWarps = 16;                         // 4 tensor-memory lane quarters x 4 quarters of a stage's weights
 constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kThreads = kDecodeThreads + 32;            // + the MMA warp
-constexpr int kARing = 2;                                // A operands in tensor memory
-constexpr int kBRing = 4;                                // B buffers in shared memory (activations run 2 stages ahead)
+#ifndef KMQ_UMMA_ARING
+#define KMQ_UMMA_ARING 6
+#endif
+constexpr int kARing = KMQ_UMMA_ARING;                   // A operands in tensor memory: the decoders may run this far ahead
+constexpr int kBRing = kARing + 2;                       // B buffers in shared memory (activations are copied 2 stages ahead)
 #ifndef KMQ_UMMA_WRING
 #define KMQ_UMMA_WRING 8
 #endif
 constexpr int kWRing = KMQ_UMMA_WRING;                   // stages of packed words in flight per thread (cp.async ring)
 constexpr int kLBO = 128;                                // bytes between core matrices that are neighbours in K
-constexpr uint32_t kWaitLimit = 1u << 20;                // polls of an mbarrier (about 20 ns apart) before giving up
+constexpr uint32_t kWaitLimit = 1u << 22;                // polls of an mbarrier before giving up (some tens of ms)
 
 template <int BITS>
 struct UGeo {
-  static constexpr int kStageK = BITS == 4 ? 128 : 256;          // weights of a row per stage
-  static constexpr int kStagesPerStep = (512 / BITS) / kStageK;  // 1, 1, 2 for b = 4, 2, 1
-  static constexpr int kThreadBytes = kStageK * BITS / 16;       // packed bytes a thread decodes per stage: 32, 32, 16
+  static constexpr int kStageK = 128;                            // weights of a row per stage
+  static constexpr int kStagesPerStep = (512 / BITS) / kStageK;  // 1, 2, 4 for b = 4, 2, 1
+  static constexpr int kThreadBytes = kStageK * BITS / 32;       // packed bytes a thread decodes per stage: 16, 8, 4
   static constexpr int kCols = kStageK / 2;                      // 32-bit columns of the A operand of a stage
   static constexpr int kKSlices = kStageK / 16;                  // MMAs per stage
   static constexpr int kSBO = (kStageK / 8) * kLBO;              // bytes between groups of 8 batch rows in a B buffer
-  static constexpr int kTmemCols = BITS == 4 ? 256 : 512;        // kARing * kCols + up to 64 columns of D, a power of two
+  static constexpr int kTmemCols = kARing * 64 + 64 <= 256 ? 256 : 512;   // kARing * kCols + up to 64 columns of D, a power of two
+  static_assert(kARing * 64 + 64 <= 512, "tensor memory has 512 columns");
   static constexpr int kTableBytes = BITS == 4 ? 4 * 16 * 128 : 0;   // b = 4: [lane quarter][entry][lane]
 };
 
@@ -107,6 +111,15 @@ __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_s
   const int bytes = valid ? 16 : 0;   // 0 source bytes: the 16 destination bytes are zero-filled
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gmem_src), "r"(bytes) : "memory");
 }
+// 8- and 4-byte variants (zero-filled when !valid)
+__device__ __forceinline__ void cp_async8(uint32_t smem_dst, const void* gmem_src, bool valid) {
+  const int bytes = valid ? 8 : 0;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(smem_dst), "l"(gmem_src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t smem_dst, const void* gmem_src, bool valid) {
+  const int bytes = valid ? 4 : 0;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_dst), "l"(gmem_src), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int PENDING>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
@@ -124,7 +137,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         : "r"(bar), "r"(parity)
         : "memory");
     if (done) return true;
-    __nanosleep(20);
   }
   return false;
 }
@@ -207,7 +219,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
   using G = UGeo<BITS>;
   using SM = USmem<BITS, NB>;
   constexpr int SPS = G::kStagesPerStep;
-  constexpr int NV = G::kThreadBytes / 16;   // 128-bit loads per thread and stage
+  constexpr int NW = G::kThreadBytes / 4;   // packed words per thread and stage: 4, 2, 1
   extern __shared__ __align__(128) unsigned char smem_raw[];
   unsigned char* const tables = smem_raw + SM::kTables;
   const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem_raw);
@@ -254,7 +266,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
 
   if (warp < kDecodeWarps) {
     // ================= decoder warps =================
-    const int q = warp & 3, kh = warp >> 2;   // tensor-memory lane quarter; which half of a stage's weights
+    const int q = warp & 3, kh = warp >> 2;   // tensor-memory lane quarter; which quarter of a stage's weights
     const int rho = 32 * q + lane;            // output row inside the CTA = tensor-memory lane
     const int64_t tiles = (N + kTileRows - 1) / kTileRows;
     const int64_t tile_id = (int64_t)blockIdx.x * (kBM / 16) + (rho >> 4);
@@ -265,14 +277,16 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
     RowState<BITS> st;
     st.init(cb + min(block_row0 + rho, N - 1) * (1 << BITS), tables + q * 2048, lane);
     // packed words of stage i: global -> this thread's slot of ring stage i % kWRing (read back by the same thread)
-    unsigned char* const w_slot = smem_raw + SM::kWords + threadIdx.x * 16;   // piece j: kDecodeThreads * 16 bytes further
-    const uint32_t w_slot_addr = smem_base + SM::kWords + threadIdx.x * 16;
+    unsigned char* const w_slot = smem_raw + SM::kWords + threadIdx.x * G::kThreadBytes;
+    const uint32_t w_slot_addr = smem_base + SM::kWords + threadIdx.x * G::kThreadBytes;
     constexpr int kWStage = kDecodeThreads * G::kThreadBytes;
     auto copy_words = [&](int i) {
       const int s = i / SPS, u = i % SPS;
-      const unsigned char* src = row_bytes + (int64_t)s * 1024 + (BITS == 1 ? 32 * u + 16 * kh : 32 * kh);
-#pragma unroll
-      for (int j = 0; j < NV; ++j) cp_async16(w_slot_addr + (i % kWRing) * kWStage + j * (kDecodeThreads * 16), src + 16 * j, has_tile);
+      // the stage's bytes of the row: [u * 64 / SPS, +64 / SPS) of its 64 bytes in the step; this thread's quarter
+      const unsigned char* src = row_bytes + (int64_t)s * 1024 + u * (64 / SPS) + kh * G::kThreadBytes;
+      if constexpr (G::kThreadBytes == 16) cp_async16(w_slot_addr + (i % kWRing) * kWStage, src, has_tile);
+      else if constexpr (G::kThreadBytes == 8) cp_async8(w_slot_addr + (i % kWRing) * kWStage, src, has_tile);
+      else cp_async4(w_slot_addr + (i % kWRing) * kWStage, src, has_tile);
     };
     // activations of stage i -> B buffer i % kBRing; piece p = (batch row m, core matrix kg), bits of p:
     // kg0 | m0..2 | kg1.. | m3..  (8 consecutive threads: 4 rows x 32 contiguous bytes)
@@ -280,8 +294,9 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
       constexpr int KGS = G::kStageK / 8;
       const uint32_t dst = b_addr + (i % kBRing) * SM::kBStageBytes;
 #pragma unroll
-      for (int j = 0; j < NB * KGS / kDecodeThreads; ++j) {
+      for (int j = 0; j < (NB * KGS + kDecodeThreads - 1) / kDecodeThreads; ++j) {
         const int p = threadIdx.x + kDecodeThreads * j;
+        if (NB * KGS % kDecodeThreads != 0 && p >= NB * KGS) break;
         const int kg = (p & 1) | (((p >> 4) & (KGS / 2 - 1)) << 1);
         const int m = ((p >> 1) & 7) | ((p / (8 * KGS)) << 3);
         const int64_t k = (int64_t)i * G::kStageK + kg * 8;
@@ -299,31 +314,34 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
       else cp_async_commit();
     }
     for (int i = 0; i < total; ++i) {
-      const int abuf = i & 1;
+      const int abuf = i % kARing;
       cp_async_wait<kWRing - 1>();   // the group of the words of stage i has landed
-      uint4 v[NV];
-#pragma unroll
-      for (int j = 0; j < NV; ++j) v[j] = *reinterpret_cast<const uint4*>(w_slot + (i % kWRing) * kWStage + j * (kDecodeThreads * 16));
+      uint32_t wv[NW];
+      if constexpr (NW == 4) {
+        const uint4 t4 = *reinterpret_cast<const uint4*>(w_slot + (i % kWRing) * kWStage);
+        wv[0] = t4.x; wv[1] = t4.y; wv[2] = t4.z; wv[3] = t4.w;
+      } else if constexpr (NW == 2) {
+        const uint2 t2 = *reinterpret_cast<const uint2*>(w_slot + (i % kWRing) * kWStage);
+        wv[0] = t2.x; wv[1] = t2.y;
+      } else {
+        wv[0] = *reinterpret_cast<const uint32_t*>(w_slot + (i % kWRing) * kWStage);
+      }
       if (i >= kARing) {
-        // the MMAs of stage i - 2 are done: A operand i % 2 and B buffer (i + 2) % 4 may be overwritten
-        ok = mbar_wait(empty_bar + 8 * abuf, ((i >> 1) - 1) & 1);
+        // the MMAs of stage i - kARing are done: A operand i % kARing and B buffer (i + 2) % kBRing may be overwritten
+        ok = mbar_wait(empty_bar + 8 * abuf, ((i / kARing) - 1) & 1);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         tc_fence_after_sync();
       }
-      // this thread's half of the stage's weights of its row -> columns kh * kCols / 2 ... of the A operand
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + abuf * G::kCols + kh * (G::kCols / 2);
+      // this thread's quarter of the stage's weights of its row -> columns kh * kCols / 4 ... of the A operand
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + abuf * G::kCols + kh * (G::kCols / 4);
+      if constexpr (BITS == 4) {
+        decode_words4_to_tmem(wv[0], wv[1], st, taddr);
+        decode_words4_to_tmem(wv[2], wv[3], st, taddr + 8);
+      } else {
+        constexpr int kColsPerWord = 16 / BITS;   // 8 or 16
 #pragma unroll
-      for (int j = 0; j < NV; ++j) {
-        const uint32_t w4[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
-        if constexpr (BITS == 4) {
-          decode_words4_to_tmem(w4[0], w4[1], st, taddr + j * 16);
-          decode_words4_to_tmem(w4[2], w4[3], st, taddr + j * 16 + 8);
-        } else {
-          constexpr int kColsPerWord = 16 / BITS;   // 8 or 16
-#pragma unroll
-          for (int jj = 0; jj < 4; ++jj) decode_word_to_tmem<BITS>(w4[jj], st, taddr + (4 * j + jj) * kColsPerWord);
-        }
+        for (int jj = 0; jj < NW; ++jj) decode_word_to_tmem<BITS>(wv[jj], st, taddr + jj * kColsPerWord);
       }
       // one group per iteration: the activations of stage i + 2 and the words of stage i + kWRing (its ring slot
       // was read above, and the decode has consumed what was read)
@@ -340,10 +358,10 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
     // ---- all MMAs done -> read the accumulator, round, store ----
     if (ok && total > 0) {
       const int last = total - 1;
-      ok = mbar_wait(empty_bar + 8 * (last & 1), (last >> 1) & 1);
+      ok = mbar_wait(empty_bar + 8 * (last % kARing), (last / kARing) & 1);
       ok = __all_sync(0xFFFFFFFFu, ok);
     }
-    if (ok) {
+    if (ok && kh < 2) {   // two warps per lane quarter split the columns
       tc_fence_after_sync();
       const int64_t n = block_row0 + rho;
 #pragma unroll
@@ -363,15 +381,15 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
         for (int j = 0; j < 8; ++j)
           if (col + j < M && n < N) y[(int64_t)(col + j) * N + n] = (uint16_t)float_to_bf16_bits(__uint_as_float(w[j]));
       }
-    } else if (lane == 0) {
+    } else if (!ok && lane == 0) {
       atomicOr(&g_device_error_flags, 1u);
     }
   } else if (lane == 0) {
     // ================= MMA warp (one thread) =================
     const uint32_t idesc = instr_desc<NB>();
     for (int i = 0; i < total; ++i) {
-      const int abuf = i & 1;
-      if (!mbar_wait(full_bar + 8 * abuf, (i >> 1) & 1)) {
+      const int abuf = i % kARing;
+      if (!mbar_wait(full_bar + 8 * abuf, (i / kARing) & 1)) {
         ok = false;
         break;
       }
@@ -424,10 +442,6 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
 
 }  // namespace
 
-#ifndef KMQ_UMMA_MIN_ROWS
-#define KMQ_UMMA_MIN_ROWS (1 << 30)
-#endif
-int linear_umma_min_rows() { return KMQ_UMMA_MIN_ROWS; }
 int linear_umma_rows_per_launch() { return 64; }
 
 cudaError_t launch_linear_umma(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,

@@ -39,6 +39,7 @@ SIGNATURES = {
     "kmq_linear_host": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr, _ptr, _ptr, _sz, _ptr]),
     "kmq_linear_static_scratch": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr]),
     "kmq_static_scratch_capacity": (_sz, []),
+    "kmq_linear_tcgen05": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _ptr]),
     "kmq_device_error_flags": (_int, [_ptr]),
     "kmq_dequant_to_bf16": (_int, [_ptr, _ptr, _ptr, _i64, _i64, _int, _int, _ptr]),
 }
@@ -168,6 +169,14 @@ def kmq_linear_static_scratch(packed, codebooks, x, y, N, K, bits, M, layout=KMQ
 
 def kmq_static_scratch_capacity() -> int:
     return lib().kmq_static_scratch_capacity()
+
+
+def kmq_linear_tcgen05(packed, codebooks, x, y, N, K, bits, M, stream=None, check=True) -> int:
+    """kmq_linear through the tcgen05 / tensor-memory kernel (tuned layout only)."""
+    st = lib().kmq_linear_tcgen05(_addr(packed), _addr(codebooks), _addr(x), _addr(y), N, K, bits, M, _stream(stream))
+    if check:
+        _check(st, "kmq_linear_tcgen05")
+    return st
 
 
 def kmq_device_error_flags() -> int:
