@@ -178,10 +178,12 @@ size_t kmq_static_scratch_capacity(void);
  * KMQ_LAYOUT_TUNED and K * bits a multiple of 128; any M >= 1 (64 batch rows
  * per launch).  This is the large-batch design the paper's roofline model
  * points to (Appendix "Theoretical model": beyond a batch of P_w * nu / 16
- * the layer is compute bound).  kmq_linear does not select it: one
- * tcgen05.mma costs at least 69 clocks whatever its N, which caps this design
- * at about 30 weights per clock and SM, and on B200 the mma.sync kernels are
- * faster up to the 64 batch rows measured (figures in the design notes).
+ * the layer is compute bound).  One tcgen05.mma (2048 weights) costs 70 to
+ * 100 clocks whatever the batch, so the time does not depend on M up to 64
+ * rows but a CTA covers 128 output rows: kmq_linear itself selects this
+ * kernel for M > 32 on shapes with enough 128-row blocks to occupy most SMs
+ * (kmq_linear_variant() then starts with "tcgen05"); this entry point forces
+ * it for any shape.
  * It needs no workspace.  Its waits on hardware barriers are bounded, see
  * kmq_device_error_flags.
  * Errors: KMQ_ERR_NULL, KMQ_ERR_BITS, KMQ_ERR_SHAPE, KMQ_ERR_ALIGN,

@@ -12,6 +12,13 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
     const bool tuned = layout == KMQ_LAYOUT_TUNED;
     p.variant = tuned ? kVariantTiled : kVariantMma;
     p.launches = (int)((M + 7) / 8);
+    if (tuned && linear_umma_selected(N, K, bits, M)) {
+      const int64_t per = linear_umma_rows_per_launch();
+      p.variant = kVariantUmma;
+      p.launches = (int)((M + per - 1) / per);
+      p.name = bits == 4 ? "tcgen05_table_b4" : bits == 2 ? "tcgen05_prmt_b2" : "tcgen05_select_b1";
+      return p;
+    }
     if (tuned && M >= linear_multi_min_rows(bits, N)) {
       const int64_t per = linear_multi_rows_per_launch(bits);
       p.variant = kVariantMulti;
@@ -47,6 +54,8 @@ cudaError_t launch_linear(const LinearPlan& plan, const uint32_t* packed, const 
   switch (plan.variant) {
     case kVariantSplit:
       return launch_linear_split(packed, cb, x, y, N, K, bits, M, workspace, plan.split_k, s);
+    case kVariantUmma:
+      return launch_linear_umma(packed, cb, x, y, N, K, bits, M, s);
     case kVariantMulti:
       return launch_linear_multi(packed, cb, x, y, N, K, bits, M, s);
     case kVariantTiled:

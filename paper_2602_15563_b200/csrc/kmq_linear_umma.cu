@@ -8,11 +8,11 @@
 //     may write is fixed by its index -- and half w / 4 of the stage's weights of that row.  In the tile-major layout
 //     the 64 bytes of a row in a step are contiguous, so the thread loads its 16 or 32 bytes directly, rebuilds the
 //     64 or 128 weights as bf16 pairs in registers and writes them with tcgen05.st into the A operand of the stage
-//     (lane = row, 32-bit column c = weights 2c, 2c + 1 of the stage).  The decoder threads also copy the
-//     activations two stages ahead (NB batch rows, zero-filled past M and past K) global -> shared with cp.async
-//     into the K-major core-matrix layout of the B operand (8 rows x 16 bytes contiguous, the next 8 weights kLBO
-//     bytes further, the next 8 rows kSBO bytes further).  When a warp's part of a stage is in place it arrives on
-//     the stage's `full` barrier;
+//     (lane = row, 32-bit column c = weights 2c, 2c + 1 of the stage).  When a warp's part of a stage is in place it
+//     arrives on the stage's `full` barrier;
+//   * a producer thread copies the activations under a stage (NB batch rows x 128, zero-filled past M and past K)
+//     with two TMA tile loads (cp.async.bulk.tensor, 64 columns = 128 bytes wide, 128-byte swizzle) into the B
+//     buffer of the stage, up to a whole ring ahead; their bytes complete the same `full` barrier;
 //   * the MMA warp waits for `full`, issues one tcgen05.mma (128 x NB x 16) per 16 weights that adds into the
 //     accumulator D[128 output rows][NB batch rows], and commits them to the stage's `empty` barrier, which the
 //     decoders wait for before they overwrite the A operand (ring of 2) and the B buffer (ring of 4).
@@ -22,6 +22,8 @@
 // Every wait on an mbarrier is bounded; a warp whose wait runs out sets bit 0 of the device error word and goes to
 // the end of the kernel (so does, after its own bounded waits, every warp that depended on it), where the tensor
 // memory is freed.
+#include <cuda.h>
+
 #include "kmq_common.cuh"
 #include "kmq_linear_variants.cuh"
 #include "kmq_mma_common.cuh"
@@ -35,18 +37,20 @@ namespace {
 constexpr int kBM = 128;                                 // output rows per CTA (rows of the MMA)
 constexpr int kDecodeWarps = 16;                         // 4 tensor-memory lane quarters x 4 quarters of a stage's weights
 constexpr int kDecodeThreads = kDecodeWarps * 32;
-constexpr int kThreads = kDecodeThreads + 32;            // + the MMA warp
+constexpr int kThreads = kDecodeThreads + 64;            // + the MMA warp + the TMA producer warp
 #ifndef KMQ_UMMA_ARING
 #define KMQ_UMMA_ARING 6
 #endif
 constexpr int kARing = KMQ_UMMA_ARING;                   // A operands in tensor memory: the decoders may run this far ahead
-constexpr int kBRing = kARing + 2;                       // B buffers in shared memory (activations are copied 2 stages ahead)
+constexpr int kBRing = kARing;                           // B buffers in shared memory, one per A operand
 #ifndef KMQ_UMMA_WRING
-#define KMQ_UMMA_WRING 8
+#define KMQ_UMMA_WRING 6
 #endif
-constexpr int kWRing = KMQ_UMMA_WRING;                   // stages of packed words in flight per thread (cp.async ring)
-constexpr int kLBO = 128;                                // bytes between core matrices that are neighbours in K
-constexpr uint32_t kWaitLimit = 1u << 22;                // polls of an mbarrier before giving up (some tens of ms)
+constexpr int kWRing = KMQ_UMMA_WRING;                   // ring of 1 KB steps of packed words per tile (cp.async), kWRing - 1 in flight
+constexpr int kWRowStride = 80;                          // a row's 64 bytes of a step, padded: lanes read consecutive rows
+constexpr int kWStepBytes = kBM * kWRowStride;
+constexpr uint32_t kWaitHintNs = 20000;                  // one try_wait on an mbarrier may park the thread this long
+constexpr uint32_t kWaitLimit = 1u << 12;                // tries before giving up (at most about 80 ms)
 
 template <int BITS>
 struct UGeo {
@@ -55,7 +59,6 @@ struct UGeo {
   static constexpr int kThreadBytes = kStageK * BITS / 32;       // packed bytes a thread decodes per stage: 16, 8, 4
   static constexpr int kCols = kStageK / 2;                      // 32-bit columns of the A operand of a stage
   static constexpr int kKSlices = kStageK / 16;                  // MMAs per stage
-  static constexpr int kSBO = (kStageK / 8) * kLBO;              // bytes between groups of 8 batch rows in a B buffer
   static constexpr int kTmemCols = kARing * 64 + 64 <= 256 ? 256 : 512;   // kARing * kCols + up to 64 columns of D, a power of two
   static_assert(kARing * 64 + 64 <= 512, "tensor memory has 512 columns");
   static constexpr int kTableBytes = BITS == 4 ? 4 * 16 * 128 : 0;   // b = 4: [lane quarter][entry][lane]
@@ -63,20 +66,33 @@ struct UGeo {
 
 template <int BITS, int NB>
 struct USmem {
-  static constexpr int kBStageBytes = NB * UGeo<BITS>::kStageK * 2;
+  static constexpr int kBHalfBytes = NB * 128;                      // NB rows x 64 activations (one TMA box)
+  static constexpr int kBStageBytes = 2 * kBHalfBytes;
   static constexpr int kB = 0;
-  static constexpr int kWords = kB + kBRing * kBStageBytes;   // ring of packed words: [stage][16-byte piece][thread]
-  static constexpr int kTables = kWords + kWRing * kDecodeThreads * UGeo<BITS>::kThreadBytes;
+  static constexpr int kWords = kB + kBRing * kBStageBytes;   // ring of packed words: [step][row][80]
+  static constexpr int kTables = kWords + kWRing * kWStepBytes;
   static constexpr int kBars = kTables + UGeo<BITS>::kTableBytes;   // full[kARing], empty[kARing]
-  static constexpr int kTmemSlot = kBars + 2 * kARing * 8;
-  static constexpr int kTotal = kTmemSlot + 16;
+  static constexpr int kTmemSlot = kBars + 2 * kARing * 8;   // then a word that a failed wait sets
+  static constexpr int kTotal = kTmemSlot + 16 + 1024;   // + room to align the base to 1024 bytes (swizzled B buffers)
 };
 
-// Shared-memory matrix descriptor: K-major, no swizzle, strides kLBO / kSBO, descriptor version of sm_100.
-template <int SBO>
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(kLBO >> 4) << 16) | ((uint64_t)(SBO >> 4) << 32) |
-         ((uint64_t)1 << 46);
+// Shared-memory matrix descriptor of a K-major operand in the 128-byte-swizzle layout TMA writes: rows of 128 bytes,
+// 8-row groups 1024 bytes apart (stride byte offset), descriptor version of sm_100, layout type 2 = 128-byte swizzle.
+// The buffer is 1024-byte aligned; 16 weights further along K = 32 bytes further in the start address.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// TMA tile load of the box at (c0, c1) of a 2-D tensor map into shared memory; its bytes complete on `bar`.
+__device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
 }
 
 // Instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, M = kBM, N = NB.
@@ -105,20 +121,10 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void async_proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src, bool valid) {
   const int bytes = valid ? 16 : 0;   // 0 source bytes: the 16 destination bytes are zero-filled
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gmem_src), "r"(bytes) : "memory");
-}
-// 8- and 4-byte variants (zero-filled when !valid)
-__device__ __forceinline__ void cp_async8(uint32_t smem_dst, const void* gmem_src, bool valid) {
-  const int bytes = valid ? 8 : 0;
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(smem_dst), "l"(gmem_src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async4(uint32_t smem_dst, const void* gmem_src, bool valid) {
-  const int bytes = valid ? 4 : 0;
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_dst), "l"(gmem_src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int PENDING>
@@ -127,14 +133,15 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-// Bounded wait for the phase of parity `parity` of an mbarrier.
+// Bounded wait for the phase of parity `parity` of an mbarrier.  try_wait parks the thread in hardware for up to the
+// hinted time instead of spinning, so waiting warps do not take issue slots from the ones that decode.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   for (uint32_t i = 0; i < kWaitLimit; ++i) {
     uint32_t done;
     asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(done)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kWaitHintNs)
         : "memory");
     if (done) return true;
   }
@@ -213,14 +220,16 @@ __device__ __forceinline__ void decode_words4_to_tmem(uint32_t w0, uint32_t w1, 
 template <int BITS, int NB>
 __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t* __restrict__ packed,
                                                                   const uint16_t* __restrict__ cb,
-                                                                  const uint16_t* __restrict__ x,
+                                                                  const __grid_constant__ CUtensorMap xmap,
                                                                   uint16_t* __restrict__ y, int64_t N, int64_t K,
                                                                   int M) {
   using G = UGeo<BITS>;
   using SM = USmem<BITS, NB>;
   constexpr int SPS = G::kStagesPerStep;
   constexpr int NW = G::kThreadBytes / 4;   // packed words per thread and stage: 4, 2, 1
-  extern __shared__ __align__(128) unsigned char smem_raw[];
+  extern __shared__ __align__(1024) unsigned char smem_unaligned[];
+  unsigned char* const smem_raw =
+      smem_unaligned + ((1024u - ((uint32_t)__cvta_generic_to_shared(smem_unaligned) & 1023u)) & 1023u);
   unsigned char* const tables = smem_raw + SM::kTables;
   const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem_raw);
   const uint32_t b_addr = smem_base + SM::kB;
@@ -235,9 +244,11 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
 
   // ---- set-up: mbarriers, tensor memory, tables ----
   if (threadIdx.x == 0) {
+    *reinterpret_cast<volatile uint32_t*>(smem_raw + SM::kTmemSlot + 4) = 0;
 #pragma unroll
     for (int i = 0; i < kARing; ++i) {
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full_bar + 8 * i), "r"(kDecodeWarps) : "memory");
+      // decoder warps + the producer's arrive-and-expect; the TMA bytes complete the same phase
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full_bar + 8 * i), "r"(kDecodeWarps + 1) : "memory");
       asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(empty_bar + 8 * i) : "memory");
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -269,91 +280,73 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
     const int q = warp & 3, kh = warp >> 2;   // tensor-memory lane quarter; which quarter of a stage's weights
     const int rho = 32 * q + lane;            // output row inside the CTA = tensor-memory lane
     const int64_t tiles = (N + kTileRows - 1) / kTileRows;
-    const int64_t tile_id = (int64_t)blockIdx.x * (kBM / 16) + (rho >> 4);
-    const bool has_tile = tile_id < tiles;    // rows of a missing tile decode zeros; they are never stored
-    // row rho % 16 of a tile owns bytes [64 (rho % 16), +64) of each 1 KB step
-    const unsigned char* __restrict__ row_bytes = reinterpret_cast<const unsigned char*>(packed) +
-                                                  (has_tile ? tile_id : 0) * (int64_t)steps * 1024 + (rho & 15) * 64;
+    // row rho % 16 of a tile owns bytes [64 (rho % 16), +64) of each 1 KB step; rows of a tile past N decode zeros
+    // and are never stored
     RowState<BITS> st;
     st.init(cb + min(block_row0 + rho, N - 1) * (1 << BITS), tables + q * 2048, lane);
-    // packed words of stage i: global -> this thread's slot of ring stage i % kWRing (read back by the same thread)
-    unsigned char* const w_slot = smem_raw + SM::kWords + threadIdx.x * G::kThreadBytes;
-    const uint32_t w_slot_addr = smem_base + SM::kWords + threadIdx.x * G::kThreadBytes;
-    constexpr int kWStage = kDecodeThreads * G::kThreadBytes;
-    auto copy_words = [&](int i) {
-      const int s = i / SPS, u = i % SPS;
-      // the stage's bytes of the row: [u * 64 / SPS, +64 / SPS) of its 64 bytes in the step; this thread's quarter
-      const unsigned char* src = row_bytes + (int64_t)s * 1024 + u * (64 / SPS) + kh * G::kThreadBytes;
-      if constexpr (G::kThreadBytes == 16) cp_async16(w_slot_addr + (i % kWRing) * kWStage, src, has_tile);
-      else if constexpr (G::kThreadBytes == 8) cp_async8(w_slot_addr + (i % kWRing) * kWStage, src, has_tile);
-      else cp_async4(w_slot_addr + (i % kWRing) * kWStage, src, has_tile);
-    };
-    // activations of stage i -> B buffer i % kBRing; piece p = (batch row m, core matrix kg), bits of p:
-    // kg0 | m0..2 | kg1.. | m3..  (8 consecutive threads: 4 rows x 32 contiguous bytes)
-    auto stage_x = [&](int i) {
-      constexpr int KGS = G::kStageK / 8;
-      const uint32_t dst = b_addr + (i % kBRing) * SM::kBStageBytes;
-#pragma unroll
-      for (int j = 0; j < (NB * KGS + kDecodeThreads - 1) / kDecodeThreads; ++j) {
-        const int p = threadIdx.x + kDecodeThreads * j;
-        if (NB * KGS % kDecodeThreads != 0 && p >= NB * KGS) break;
-        const int kg = (p & 1) | (((p >> 4) & (KGS / 2 - 1)) << 1);
-        const int m = ((p >> 1) & 7) | ((p / (8 * KGS)) << 3);
-        const int64_t k = (int64_t)i * G::kStageK + kg * 8;
-        const bool valid = m < M && k < K;
-        cp_async16(dst + (m >> 3) * G::kSBO + kg * kLBO + (m & 7) * 16, x + (valid ? (int64_t)m * K + k : 0), valid);
-      }
+    // packed words: whole 1 KB steps of the CTA's 8 tiles, global -> shared, coalesced (thread j copies 16-byte piece
+    // j % 64 of tile j / 64 = piece j % 4 of row j / 4), one cp.async group per step, kWRing - 1 steps in flight
+    const unsigned char* const w_row = smem_raw + SM::kWords + rho * kWRowStride + kh * G::kThreadBytes;
+    const int cj = threadIdx.x;
+    const int64_t c_tile = (int64_t)blockIdx.x * (kBM / 16) + (cj >> 6);
+    const unsigned char* const c_src =
+        reinterpret_cast<const unsigned char*>(packed) + (c_tile < tiles ? c_tile : 0) * (int64_t)steps * 1024 + (cj & 63) * 16;
+    const uint32_t c_dst = smem_base + SM::kWords + (cj >> 2) * kWRowStride + (cj & 3) * 16;
+    auto copy_step = [&](int s) {
+      if (s < steps) cp_async16(c_dst + (s % kWRing) * kWStepBytes, c_src + (int64_t)s * 1024, c_tile < tiles);
       cp_async_commit();
     };
-
-    // prologue: kWRing groups; group d holds the words of stage d and, for d < 2, the activations of stage d
+    volatile uint32_t* const fail_word = reinterpret_cast<volatile uint32_t*>(smem_raw + SM::kTmemSlot + 4);
 #pragma unroll 1
-    for (int d = 0; d < kWRing; ++d) {
-      if (d < total) copy_words(d);
-      if (d < 2 && d < total) stage_x(d);
-      else cp_async_commit();
-    }
-    for (int i = 0; i < total; ++i) {
-      const int abuf = i % kARing;
-      cp_async_wait<kWRing - 1>();   // the group of the words of stage i has landed
-      uint32_t wv[NW];
-      if constexpr (NW == 4) {
-        const uint4 t4 = *reinterpret_cast<const uint4*>(w_slot + (i % kWRing) * kWStage);
-        wv[0] = t4.x; wv[1] = t4.y; wv[2] = t4.z; wv[3] = t4.w;
-      } else if constexpr (NW == 2) {
-        const uint2 t2 = *reinterpret_cast<const uint2*>(w_slot + (i % kWRing) * kWStage);
-        wv[0] = t2.x; wv[1] = t2.y;
-      } else {
-        wv[0] = *reinterpret_cast<const uint32_t*>(w_slot + (i % kWRing) * kWStage);
+    for (int d = 0; d < kWRing - 1; ++d) copy_step(d);
+    int i = 0;   // stage
+    for (int s = 0; s < steps; ++s) {
+      cp_async_wait<kWRing - 2>();   // this thread's piece of step s has landed
+      // every decoder thread's piece of step s has landed, and every one is done with step s - 1
+      asm volatile("bar.sync 1, %0;" ::"n"(kDecodeThreads) : "memory");
+      if (*fail_word) {   // some warp's wait ran out: all decoders leave together
+        ok = false;
+        break;
       }
-      if (i >= kARing) {
-        // the MMAs of stage i - kARing are done: A operand i % kARing and B buffer (i + 2) % kBRing may be overwritten
-        ok = mbar_wait(empty_bar + 8 * abuf, ((i / kARing) - 1) & 1);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) break;
-        tc_fence_after_sync();
-      }
-      // this thread's quarter of the stage's weights of its row -> columns kh * kCols / 4 ... of the A operand
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + abuf * G::kCols + kh * (G::kCols / 4);
-      if constexpr (BITS == 4) {
-        decode_words4_to_tmem(wv[0], wv[1], st, taddr);
-        decode_words4_to_tmem(wv[2], wv[3], st, taddr + 8);
-      } else {
-        constexpr int kColsPerWord = 16 / BITS;   // 8 or 16
+      copy_step(s + kWRing - 1);     // into the slot of step s - 1
+      const unsigned char* const w_step = w_row + (s % kWRing) * kWStepBytes;
 #pragma unroll
-        for (int jj = 0; jj < NW; ++jj) decode_word_to_tmem<BITS>(wv[jj], st, taddr + jj * kColsPerWord);
+      for (int u = 0; u < SPS; ++u, ++i) {
+        const int abuf = i % kARing;
+        // the stage's bytes of the row: [u * 64 / SPS, +64 / SPS) of its 64 bytes in the step; this thread's quarter
+        uint32_t wv[NW];
+        if constexpr (NW == 4) {
+          const uint4 t4 = *reinterpret_cast<const uint4*>(w_step + u * (64 / SPS));
+          wv[0] = t4.x; wv[1] = t4.y; wv[2] = t4.z; wv[3] = t4.w;
+        } else if constexpr (NW == 2) {
+          const uint2 t2 = *reinterpret_cast<const uint2*>(w_step + u * (64 / SPS));
+          wv[0] = t2.x; wv[1] = t2.y;
+        } else {
+          wv[0] = *reinterpret_cast<const uint32_t*>(w_step + u * (64 / SPS));
+        }
+        if (ok && i >= kARing) {
+          // the MMAs of stage i - kARing are done: A operand i % kARing may be overwritten
+          ok = mbar_wait(empty_bar + 8 * abuf, ((i / kARing) - 1) & 1);
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) *fail_word = 1;
+          tc_fence_after_sync();
+        }
+        if (!ok) continue;   // up to the next barrier, where all decoders leave
+        // this thread's quarter of the stage's weights of its row -> columns kh * kCols / 4 ... of the A operand
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + abuf * G::kCols + kh * (G::kCols / 4);
+        if constexpr (BITS == 4) {
+          decode_words4_to_tmem(wv[0], wv[1], st, taddr);
+          decode_words4_to_tmem(wv[2], wv[3], st, taddr + 8);
+        } else {
+          constexpr int kColsPerWord = 16 / BITS;   // 8 or 16
+#pragma unroll
+          for (int jj = 0; jj < NW; ++jj) decode_word_to_tmem<BITS>(wv[jj], st, taddr + jj * kColsPerWord);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full_bar + 8 * abuf);
       }
-      // one group per iteration: the activations of stage i + 2 and the words of stage i + kWRing (its ring slot
-      // was read above, and the decode has consumed what was read)
-      if (i + kWRing < total) copy_words(i + kWRing);
-      if (i + 2 < total) stage_x(i + 2);
-      else cp_async_commit();
-      cp_async_wait<2>();   // the group with the activations of stage i has landed
-      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-      async_proxy_fence();   // the copies into shared memory become visible to the tensor core's reads
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(full_bar + 8 * abuf);
     }
     // ---- all MMAs done -> read the accumulator, round, store ----
     if (ok && total > 0) {
@@ -384,7 +377,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
     } else if (!ok && lane == 0) {
       atomicOr(&g_device_error_flags, 1u);
     }
-  } else if (lane == 0) {
+  } else if (warp == kDecodeWarps && lane == 0) {
     // ================= MMA warp (one thread) =================
     const uint32_t idesc = instr_desc<NB>();
     for (int i = 0; i < total; ++i) {
@@ -394,12 +387,25 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
         break;
       }
       tc_fence_after_sync();
-      const uint32_t b_stage = b_addr + (i % kBRing) * SM::kBStageBytes;
+      const uint32_t b_stage = b_addr + abuf * SM::kBStageBytes;
 #pragma unroll
-      for (int ks = 0; ks < G::kKSlices; ++ks)
-        umma_bf16(tmem_d, tmem_base + abuf * G::kCols + ks * 8, smem_desc<G::kSBO>(b_stage + ks * 2 * kLBO), idesc,
-                  (i | ks) != 0);
+      for (int ks = 0; ks < G::kKSlices; ++ks)   // 16 activations = 32 bytes further inside a 128-byte row
+        umma_bf16(tmem_d, tmem_base + abuf * G::kCols + ks * 8,
+                  smem_desc_sw128(b_stage + (ks >> 2) * SM::kBHalfBytes + (ks & 3) * 32), idesc, (i | ks) != 0);
       umma_commit(empty_bar + 8 * abuf);
+    }
+    if (!ok) atomicOr(&g_device_error_flags, 1u);
+  } else if (warp == kDecodeWarps + 1 && lane == 0) {
+    // ================= TMA producer (one thread) =================
+    for (int j = 0; j < total; ++j) {
+      const int buf = j % kARing;
+      if (j >= kARing && !mbar_wait(empty_bar + 8 * buf, ((j / kARing) - 1) & 1)) {   // the MMAs that read the buffer
+        ok = false;
+        break;
+      }
+      mbar_expect_tx(full_bar + 8 * buf, SM::kBStageBytes);
+      tma_load_2d(b_addr + buf * SM::kBStageBytes, &xmap, j * G::kStageK, 0, full_bar + 8 * buf);
+      tma_load_2d(b_addr + buf * SM::kBStageBytes + SM::kBHalfBytes, &xmap, j * G::kStageK + 64, 0, full_bar + 8 * buf);
     }
     if (!ok) atomicOr(&g_device_error_flags, 1u);
   }
@@ -414,6 +420,38 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
 
 namespace {
 
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up once through the runtime (no link against the driver library).
+EncodeTiledFn encode_tiled() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// x as a 2-D tensor [M rows][K] of bf16; boxes of NB rows x 64 columns (128 bytes) land in shared memory with the
+// 128-byte swizzle; rows past M and columns past K read as zero.
+template <int NB>
+bool make_x_map(CUtensorMap* map, const uint16_t* x, int64_t K, int M) {
+  EncodeTiledFn enc = encode_tiled();
+  if (!enc) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)NB};
+  const cuuint32_t elem[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t*>(x), dims, strides, box, elem,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BITS, int NB>
 cudaError_t launch_nb(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N, int64_t K,
                       int M, cudaStream_t s) {
@@ -426,8 +464,10 @@ cudaError_t launch_nb(const uint32_t* packed, const uint16_t* cb, const uint16_t
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
+  CUtensorMap xmap;
+  if (!make_x_map<NB>(&xmap, x, K, M)) return cudaErrorInvalidValue;
   const unsigned grid = (unsigned)((N + kBM - 1) / kBM);
-  linear_umma_kernel<BITS, NB><<<grid, kThreads, smem, s>>>(packed, cb, x, y, N, K, M);
+  linear_umma_kernel<BITS, NB><<<grid, kThreads, smem, s>>>(packed, cb, xmap, y, N, K, M);
   return cudaGetLastError();
 }
 
@@ -443,6 +483,17 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
 }  // namespace
 
 int linear_umma_rows_per_launch() { return 64; }
+
+// The tensor core issues one tcgen05.mma (2048 weights) per 70-100 clocks whatever the batch, so the kernel's time
+// does not depend on M up to 64 rows, but a CTA covers 128 output rows: it pays when the batch is large and there
+// are enough 128-row blocks to occupy most SMs.  Measured: 16384 x 3072, b = 2: 18.5 us for any M <= 64 against
+// 18.5 / 28.5 / 31.6 us of the multi-tile kernel at M = 32 / 40 / 64; 12288 x 4096, M = 64: 22.7 against 38.9 us;
+// 8192 x 8192 (64 blocks), M = 64: 38.9 against 36.0 us.
+bool linear_umma_selected(int64_t N, int64_t K, int bits, int64_t M) {
+  const DeviceInfo* di = device_info();
+  if (!di || M <= 32 || (K * bits) % 128 != 0) return false;
+  return (N + kBM - 1) / kBM >= (int64_t)di->sm_count * 5 / 8;
+}
 
 cudaError_t launch_linear_umma(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                int64_t K, int bits, int64_t M, cudaStream_t s) {

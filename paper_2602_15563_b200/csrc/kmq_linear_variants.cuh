@@ -10,6 +10,8 @@ enum LinearVariant : int {
   kVariantTiled = 2,     // tuned (tile-major) layout: tensor-core GEMV with coalesced 1 KB steps, small batches (M <= 8)
   kVariantMulti = 3,     // tuned layout, M >= linear_multi_min_rows(): 32 or 64 rows per CTA share the staged
                          // activations, one decode feeds up to 8 MMAs
+  kVariantUmma = 5,      // tuned layout, M > 32 and enough 128-row blocks to fill the SMs: tcgen05.mma, weights
+                         // dequantised into tensor memory
   kVariantSplit = 4,     // tuned layout, M <= 8, more tiles than resident CTAs: equal step ranges + fix-up (scratch)
 };
 
@@ -30,6 +32,7 @@ int linear_multi_rows_per_launch(int bits);
 int linear_multi_min_rows(int bits, int64_t N);   // smallest batch routed to the multi-tile kernel
 cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                 int64_t K, int bits, int64_t M, cudaStream_t s);
+bool linear_umma_selected(int64_t N, int64_t K, int bits, int64_t M);   // kmq_linear's choice of the tcgen05 kernel
 int linear_umma_rows_per_launch();
 cudaError_t launch_linear_umma(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                int64_t K, int bits, int64_t M, cudaStream_t s);

@@ -80,6 +80,15 @@ def test_config3_decoder_linear_set(name, M):
     run_case(3, name, 2, M, check_dequant=(M == 1))
 
 
+def test_large_batch_on_many_rows_goes_through_tcgen05():
+    """16384 rows are 128 blocks of 128: from 33 batch rows on kmq_linear picks the tensor-memory kernel there."""
+    assert kmq.kmq_linear_variant(16384, 3072, 2, 64, T).startswith("tcgen05")
+    assert kmq.kmq_linear_num_launches(16384, 3072, 2, 64, T) == 1
+    assert kmq.kmq_workspace_bytes(16384, 3072, 2, 64, T) == 0
+    run_case(3, "gate_up", 2, 64, check_dequant=False)
+    assert kmq.kmq_device_error_flags() == 0
+
+
 @pytest.mark.parametrize("M", (1, 2, 4, 8, 16, 32, 64))
 def test_config4_batch_sweep_8192(M):
     run_case(4, "square8192", 2, M, check_dequant=(M == 1))
