@@ -133,6 +133,29 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// All threads of all CTAs of the cluster.
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The shared::cluster address of CTA 0's copy of this CTA's shared-memory address `saddr`.
+__device__ __forceinline__ uint32_t map_to_rank0(uint32_t saddr) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(r) : "r"(saddr));
+  return r;
+}
+// 8 consecutive columns of this thread's lane of the accumulator (zeros when nothing was accumulated)
+__device__ __forceinline__ void load_acc8(uint32_t (&w)[8], uint32_t taddr, bool valid) {
+  if (valid) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) w[j] = 0;
+  }
+}
+
 // Bounded wait for the phase of parity `parity` of an mbarrier.  try_wait parks the thread in hardware for up to the
 // hinted time instead of spinning, so waiting warps do not take issue slots from the ones that decode.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
@@ -240,7 +263,11 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
   const int64_t block_row0 = (int64_t)blockIdx.x * kBM;
   const int chunks = (int)(K / (128 / BITS));   // 16-byte chunks per row
   const int steps = (chunks + 3) >> 2;          // the layout pads every row to whole steps of 64 bytes
-  const int total = steps * SPS;                // stages
+  // K is split over the gridDim.y CTAs of a cluster (same output rows): rank r takes steps [s_begin, s_end)
+  const int ksplit = gridDim.y, rank = blockIdx.y;
+  const int s_begin = (int)((int64_t)steps * rank / ksplit), s_end = (int)((int64_t)steps * (rank + 1) / ksplit);
+  const int my_steps = s_end - s_begin;
+  const int total = my_steps * SPS;             // stages of this CTA
 
   // ---- set-up: mbarriers, tensor memory, tables ----
   if (threadIdx.x == 0) {
@@ -290,17 +317,18 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
     const int cj = threadIdx.x;
     const int64_t c_tile = (int64_t)blockIdx.x * (kBM / 16) + (cj >> 6);
     const unsigned char* const c_src =
-        reinterpret_cast<const unsigned char*>(packed) + (c_tile < tiles ? c_tile : 0) * (int64_t)steps * 1024 + (cj & 63) * 16;
+        reinterpret_cast<const unsigned char*>(packed) + ((c_tile < tiles ? c_tile : 0) * (int64_t)steps + s_begin) * 1024 +
+        (cj & 63) * 16;
     const uint32_t c_dst = smem_base + SM::kWords + (cj >> 2) * kWRowStride + (cj & 3) * 16;
     auto copy_step = [&](int s) {
-      if (s < steps) cp_async16(c_dst + (s % kWRing) * kWStepBytes, c_src + (int64_t)s * 1024, c_tile < tiles);
+      if (s < my_steps) cp_async16(c_dst + (s % kWRing) * kWStepBytes, c_src + (int64_t)s * 1024, c_tile < tiles);
       cp_async_commit();
     };
     volatile uint32_t* const fail_word = reinterpret_cast<volatile uint32_t*>(smem_raw + SM::kTmemSlot + 4);
 #pragma unroll 1
     for (int d = 0; d < kWRing - 1; ++d) copy_step(d);
     int i = 0;   // stage
-    for (int s = 0; s < steps; ++s) {
+    for (int s = 0; s < my_steps; ++s) {
       cp_async_wait<kWRing - 2>();   // this thread's piece of step s has landed
       // every decoder thread's piece of step s has landed, and every one is done with step s - 1
       asm volatile("bar.sync 1, %0;" ::"n"(kDecodeThreads) : "memory");
@@ -348,35 +376,13 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
         if (lane == 0) mbar_arrive(full_bar + 8 * abuf);
       }
     }
-    // ---- all MMAs done -> read the accumulator, round, store ----
+    // ---- wait until all MMAs of this CTA are done ----
     if (ok && total > 0) {
       const int last = total - 1;
       ok = mbar_wait(empty_bar + 8 * (last % kARing), (last / kARing) & 1);
       ok = __all_sync(0xFFFFFFFFu, ok);
     }
-    if (ok && kh < 2) {   // two warps per lane quarter split the columns
-      tc_fence_after_sync();
-      const int64_t n = block_row0 + rho;
-#pragma unroll
-      for (int c0 = 0; c0 < NB / 2; c0 += 8) {
-        const int col = kh * (NB / 2) + c0;   // the two warps of a lane quarter split the columns
-        uint32_t w[8];
-        if (total > 0) {
-          asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                       : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
-                       : "r"(tmem_d + ((uint32_t)(q * 32) << 16) + col));
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        } else {
-#pragma unroll
-          for (int j = 0; j < 8; ++j) w[j] = 0;
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (col + j < M && n < N) y[(int64_t)(col + j) * N + n] = (uint16_t)float_to_bf16_bits(__uint_as_float(w[j]));
-      }
-    } else if (!ok && lane == 0) {
-      atomicOr(&g_device_error_flags, 1u);
-    }
+    if (!ok && lane == 0) atomicOr(&g_device_error_flags, 1u);
   } else if (warp == kDecodeWarps && lane == 0) {
     // ================= MMA warp (one thread) =================
     const uint32_t idesc = instr_desc<NB>();
@@ -404,10 +410,52 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
         break;
       }
       mbar_expect_tx(full_bar + 8 * buf, SM::kBStageBytes);
-      tma_load_2d(b_addr + buf * SM::kBStageBytes, &xmap, j * G::kStageK, 0, full_bar + 8 * buf);
-      tma_load_2d(b_addr + buf * SM::kBStageBytes + SM::kBHalfBytes, &xmap, j * G::kStageK + 64, 0, full_bar + 8 * buf);
+      const int k0 = (s_begin * SPS + j) * G::kStageK;
+      tma_load_2d(b_addr + buf * SM::kBStageBytes, &xmap, k0, 0, full_bar + 8 * buf);
+      tma_load_2d(b_addr + buf * SM::kBStageBytes + SM::kBHalfBytes, &xmap, k0 + 64, 0, full_bar + 8 * buf);
     }
     if (!ok) atomicOr(&g_device_error_flags, 1u);
+  }
+  // ---- accumulators of the cluster -> rank 0 -> bf16 ----
+  // Rank r > 0 hands its accumulator to rank 0 through rank 0's shared memory (the ring of packed words, free once
+  // every CTA of the cluster has left its main loop): [r - 1][batch row][output row] floats.
+  __syncwarp();
+  if (ksplit > 1) cluster_sync();
+  const bool reader = warp < kDecodeWarps && (warp >> 2) < 2 && ok;   // two warps per lane quarter split the columns
+  if (reader) {
+    const int q = warp & 3, kh = warp >> 2, rho = 32 * q + lane;
+    tc_fence_after_sync();
+    if (rank != 0) {
+      const uint32_t remote = map_to_rank0(smem_base + SM::kWords) + (uint32_t)(rank - 1) * (NB * kBM * 4);
+#pragma unroll
+      for (int c0 = 0; c0 < NB / 2; c0 += 8) {
+        const int col = kh * (NB / 2) + c0;
+        uint32_t w[8];
+        load_acc8(w, tmem_d + ((uint32_t)(q * 32) << 16) + col, total > 0);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(remote + ((col + j) * kBM + rho) * 4), "r"(w[j]) : "memory");
+      }
+    }
+  }
+  __syncwarp();
+  if (ksplit > 1) cluster_sync();
+  if (reader && rank == 0) {
+    const int q = warp & 3, kh = warp >> 2, rho = 32 * q + lane;
+    const int64_t n = block_row0 + rho;
+    const float* const partial = reinterpret_cast<const float*>(smem_raw + SM::kWords);
+#pragma unroll
+    for (int c0 = 0; c0 < NB / 2; c0 += 8) {
+      const int col = kh * (NB / 2) + c0;
+      uint32_t w[8];
+      load_acc8(w, tmem_d + ((uint32_t)(q * 32) << 16) + col, total > 0);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float v = __uint_as_float(w[j]);
+        for (int r = 1; r < ksplit; ++r) v += partial[((r - 1) * NB + col + j) * kBM + rho];   // fixed order
+        if (col + j < M && n < N) y[(int64_t)(col + j) * N + n] = (uint16_t)float_to_bf16_bits(v);
+      }
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -464,11 +512,24 @@ cudaError_t launch_nb(const uint32_t* packed, const uint16_t* cb, const uint16_t
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
+  static_assert(NB * kBM * 4 <= kWRing * kWStepBytes, "the partial accumulator of the second CTA must fit the words ring");
   CUtensorMap xmap;
   if (!make_x_map<NB>(&xmap, x, K, M)) return cudaErrorInvalidValue;
-  const unsigned grid = (unsigned)((N + kBM - 1) / kBM);
-  linear_umma_kernel<BITS, NB><<<grid, kThreads, smem, s>>>(packed, cb, xmap, y, N, K, M);
-  return cudaGetLastError();
+  const unsigned blocks = (unsigned)((N + kBM - 1) / kBM);
+  const int ksplit = linear_umma_ksplit(N, K, BITS);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks, (unsigned)ksplit);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = (unsigned)ksplit;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = ksplit > 1 ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, linear_umma_kernel<BITS, NB>, packed, cb, xmap, y, N, K, M);
 }
 
 template <int BITS>
@@ -484,6 +545,14 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
 
 int linear_umma_rows_per_launch() { return 64; }
 
+// CTAs per 128-row block: K is split over a cluster of 2 (partial sums meet in CTA 0's shared memory) while the
+// blocks alone would leave at least half of the SMs idle and each half still has a few steps.
+int linear_umma_ksplit(int64_t N, int64_t K, int bits) {
+  const DeviceInfo* di = device_info();
+  const int64_t blocks = (N + kBM - 1) / kBM, steps = (K * bits / 128 + 3) / 4;
+  return (di && blocks * 2 <= di->sm_count && steps >= 8) ? 2 : 1;
+}
+
 // The tensor core issues one tcgen05.mma (2048 weights) per 70-100 clocks whatever the batch, so the kernel's time
 // does not depend on M up to 64 rows, but a CTA covers 128 output rows: it pays when the batch is large and there
 // are enough 128-row blocks to occupy most SMs.  Measured: 16384 x 3072, b = 2: 18.5 us for any M <= 64 against
@@ -492,7 +561,7 @@ int linear_umma_rows_per_launch() { return 64; }
 bool linear_umma_selected(int64_t N, int64_t K, int bits, int64_t M) {
   const DeviceInfo* di = device_info();
   if (!di || M <= 32 || (K * bits) % 128 != 0) return false;
-  return (N + kBM - 1) / kBM >= (int64_t)di->sm_count * 5 / 8;
+  return (N + kBM - 1) / kBM * linear_umma_ksplit(N, K, bits) >= (int64_t)di->sm_count * 5 / 8;
 }
 
 cudaError_t launch_linear_umma(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
