@@ -63,7 +63,7 @@ CONFIG_ID = {"config2": 2, "config3_m1": 3, "config3_m8": 3, "config4": 4, "conf
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel,
 # from the ncu capture summarised under profiles/ (None = not captured yet).
 NCU_TRAFFIC_BYTES = {                      # (workload, bits, M) -> bytes; profiles/kmq_linear_tiled_config2_ncu_full.md
-    ("config2", 1, 1): 2141184, ("config2", 2, 1): 4249088, ("config2", 4, 1): 8538624,
+    ("config2", 1, 1): 2141184, ("config2", 2, 1): 4249088, ("config2", 4, 1): 8539392,
 }
 
 
