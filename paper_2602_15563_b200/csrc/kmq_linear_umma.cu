@@ -1,27 +1,30 @@
-// kmq_linear on the tuned (tile-major) layout for batches of 16 rows and more: the 5th-generation tensor core
-// (tcgen05.mma) multiplies dequantised bf16 weights, held in tensor memory, with the activations in shared memory;
-// the accumulator lives in tensor memory too.
+// kmq_linear on the tuned (tile-major) layout for large batches: the 5th-generation tensor core (tcgen05.mma)
+// multiplies dequantised bf16 weights, held in tensor memory, with the activations in shared memory; the accumulator
+// lives in tensor memory too.
 //
-// One CTA owns 128 output rows (8 tiles of 16) and walks K in stages of 256 (b = 4: 128) weights per row.  Its 8
-// decoder warps and one MMA warp meet only through mbarriers:
-//   * decoder thread (warp w, lane l) owns output row 32 (w % 4) + l of the CTA -- the tensor-memory lane a warp
-//     may write is fixed by its index -- and half w / 4 of the stage's weights of that row.  In the tile-major layout
-//     the 64 bytes of a row in a step are contiguous, so the thread loads its 16 or 32 bytes directly, rebuilds the
-//     64 or 128 weights as bf16 pairs in registers and writes them with tcgen05.st into the A operand of the stage
-//     (lane = row, 32-bit column c = weights 2c, 2c + 1 of the stage).  When a warp's part of a stage is in place it
-//     arrives on the stage's `full` barrier;
-//   * a producer thread copies the activations under a stage (NB batch rows x 128, zero-filled past M and past K)
+// One CTA owns 128 output rows (8 tiles of 16) and walks its share of K in stages of 128 weights per row.  Its 16
+// decoder warps, one MMA warp and one TMA producer warp meet only through mbarriers:
+//   * the decoder threads copy the packed words of the CTA's 8 tiles, one 1 KB step per tile at a time, global ->
+//     shared with coalesced cp.async (ring of kWRing steps, rows padded to 80 bytes; one named barrier per step).
+//     Decoder thread (warp w, lane l) owns output row 32 (w % 4) + l of the CTA -- the tensor-memory lane a warp may
+//     write is fixed by its index -- and quarter w / 4 of each stage's weights of that row: it reads its 4..16 bytes
+//     from the ring, rebuilds the 32 weights as bf16 pairs in registers and writes them with tcgen05.st into the A
+//     operand of the stage (lane = row, 32-bit column c = weights 2c, 2c + 1 of the stage; ring of kARing stages).
+//     When a warp's part of a stage is in place it arrives on the stage's `full` barrier;
+//   * the producer thread copies the activations under a stage (NB batch rows x 128, zero-filled past M and past K)
 //     with two TMA tile loads (cp.async.bulk.tensor, 64 columns = 128 bytes wide, 128-byte swizzle) into the B
 //     buffer of the stage, up to a whole ring ahead; their bytes complete the same `full` barrier;
-//   * the MMA warp waits for `full`, issues one tcgen05.mma (128 x NB x 16) per 16 weights that adds into the
-//     accumulator D[128 output rows][NB batch rows], and commits them to the stage's `empty` barrier, which the
-//     decoders wait for before they overwrite the A operand (ring of 2) and the B buffer (ring of 4).
-// At the end the decoder warps read the accumulator with tcgen05.ld (lane = output row, column = batch row), round
-// to bf16 and store.
+//   * the MMA thread waits for `full`, issues 8 tcgen05.mma (128 x NB x 16 each) that add into the accumulator
+//     D[128 output rows][NB batch rows], and commits them to the stage's `empty` barrier, which the decoders and the
+//     producer wait for before they overwrite the A operand and the B buffer.
+// When the 128-row blocks alone would leave half of the SMs idle, K is split over a cluster of 2 CTAs: each
+// accumulates its half, CTA 1 writes its accumulator into CTA 0's shared memory (st.shared::cluster between two
+// cluster barriers), CTA 0 adds the two in a fixed order.  At the end the decoder warps read the accumulator with
+// tcgen05.ld (lane = output row, column = batch row), round to bf16 and store.
 //
 // Every wait on an mbarrier is bounded; a warp whose wait runs out sets bit 0 of the device error word and goes to
-// the end of the kernel (so does, after its own bounded waits, every warp that depended on it), where the tensor
-// memory is freed.
+// the end of the kernel (so does, after its own bounded waits, every warp that depended on it); every thread still
+// takes part in the cluster barriers and the final CTA barrier, after which the tensor memory is freed.
 #include <cuda.h>
 
 #include "kmq_common.cuh"
@@ -109,6 +112,15 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_tmem, uint
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       :
       : "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// the same with the accumulate flag fixed to true
+__device__ __forceinline__ void umma_bf16_acc(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.eq.u32 p, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      :
+      : "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
       : "memory");
 }
 __device__ __forceinline__ void tmem_store8(uint32_t taddr, const uint32_t (&v)[8]) {
@@ -385,20 +397,39 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
     if (!ok && lane == 0) atomicOr(&g_device_error_flags, 1u);
   } else if (warp == kDecodeWarps && lane == 0) {
     // ================= MMA warp (one thread) =================
+    // The issuing thread is blocked for about 70 clocks per tcgen05.mma and runs everything in between serially, so
+    // the per-instruction work is kept to one add: descriptors differ only in their low word.
     const uint32_t idesc = instr_desc<NB>();
+    const uint64_t desc0 = smem_desc_sw128(b_addr);
+    const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
+    uint32_t desc_lo = (uint32_t)desc0, a_tmem = tmem_base, bar_off = 0;   // of the current stage's buffer
+    int abuf = 0;
+    uint32_t parity = 0;
     for (int i = 0; i < total; ++i) {
-      const int abuf = i % kARing;
-      if (!mbar_wait(full_bar + 8 * abuf, (i / kARing) & 1)) {
+      if (!mbar_wait(full_bar + bar_off, parity)) {
         ok = false;
         break;
       }
       tc_fence_after_sync();
-      const uint32_t b_stage = b_addr + abuf * SM::kBStageBytes;
 #pragma unroll
-      for (int ks = 0; ks < G::kKSlices; ++ks)   // 16 activations = 32 bytes further inside a 128-byte row
-        umma_bf16(tmem_d, tmem_base + abuf * G::kCols + ks * 8,
-                  smem_desc_sw128(b_stage + (ks >> 2) * SM::kBHalfBytes + (ks & 3) * 32), idesc, (i | ks) != 0);
-      umma_commit(empty_bar + 8 * abuf);
+      for (int ks = 0; ks < G::kKSlices; ++ks) {   // 16 activations = 32 bytes further inside a 128-byte row
+        const uint32_t lo = desc_lo + (ks >> 2) * (SM::kBHalfBytes >> 4) + (ks & 3) * 2;
+        const uint64_t b_desc = ((uint64_t)desc_hi << 32) | lo;
+        if (ks == 0) umma_bf16(tmem_d, a_tmem, b_desc, idesc, i != 0);
+        else umma_bf16_acc(tmem_d, a_tmem + ks * 8, b_desc, idesc);
+      }
+      umma_commit(empty_bar + bar_off);
+      if (++abuf == kARing) {
+        abuf = 0;
+        parity ^= 1;
+        desc_lo = (uint32_t)desc0;
+        a_tmem = tmem_base;
+        bar_off = 0;
+      } else {
+        desc_lo += SM::kBStageBytes >> 4;
+        a_tmem += G::kCols;
+        bar_off += 8;
+      }
     }
     if (!ok) atomicOr(&g_device_error_flags, 1u);
   } else if (warp == kDecodeWarps + 1 && lane == 0) {
