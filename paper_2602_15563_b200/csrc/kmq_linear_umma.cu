@@ -209,7 +209,7 @@ struct RowState<4> {
 };
 
 // One packed word of a row -> bf16 pairs in the order of k, written to consecutive columns of the row's
-// tensor-memory lane starting at `taddr`.  Returns the number of columns written (weights per word / 2).
+// tensor-memory lane starting at `taddr` (8 columns at b = 2, 16 at b = 1).
 template <int BITS>
 __device__ __forceinline__ void decode_word_to_tmem(uint32_t w, const RowState<BITS>& st, uint32_t taddr) {
   if constexpr (BITS == 2) {
