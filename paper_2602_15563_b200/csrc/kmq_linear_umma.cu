@@ -155,16 +155,22 @@ __device__ __forceinline__ uint32_t map_to_rank0(uint32_t saddr) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(r) : "r"(saddr));
   return r;
 }
-// 8 consecutive columns of this thread's lane of the accumulator (zeros when nothing was accumulated)
-__device__ __forceinline__ void load_acc8(uint32_t (&w)[8], uint32_t taddr, bool valid) {
+// This thread's lane of the accumulator, columns [col0, col0 + NC): all loads are issued before the one wait
+// (zeros when nothing was accumulated).
+template <int NC>
+__device__ __forceinline__ void load_acc(uint32_t (&w)[NC], uint32_t taddr, bool valid) {
+  static_assert(NC % 8 == 0, "whole groups of 8 columns");
   if (valid) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
-                 : "r"(taddr));
+#pragma unroll
+    for (int c = 0; c < NC; c += 8)
+      asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                   : "=r"(w[c + 0]), "=r"(w[c + 1]), "=r"(w[c + 2]), "=r"(w[c + 3]), "=r"(w[c + 4]), "=r"(w[c + 5]),
+                     "=r"(w[c + 6]), "=r"(w[c + 7])
+                   : "r"(taddr + c));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
   } else {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) w[j] = 0;
+    for (int j = 0; j < NC; ++j) w[j] = 0;
   }
 }
 
@@ -458,15 +464,12 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
     tc_fence_after_sync();
     if (rank != 0) {
       const uint32_t remote = map_to_rank0(smem_base + SM::kWords) + (uint32_t)(rank - 1) * (NB * kBM * 4);
+      const int col0 = kh * (NB / 2);
+      uint32_t w[NB / 2];
+      load_acc<NB / 2>(w, tmem_d + ((uint32_t)(q * 32) << 16) + col0, total > 0);
 #pragma unroll
-      for (int c0 = 0; c0 < NB / 2; c0 += 8) {
-        const int col = kh * (NB / 2) + c0;
-        uint32_t w[8];
-        load_acc8(w, tmem_d + ((uint32_t)(q * 32) << 16) + col, total > 0);
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(remote + ((col + j) * kBM + rho) * 4), "r"(w[j]) : "memory");
-      }
+      for (int j = 0; j < NB / 2; ++j)
+        asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(remote + ((col0 + j) * kBM + rho) * 4), "r"(w[j]) : "memory");
     }
   }
   __syncwarp();
@@ -475,17 +478,14 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
     const int q = warp & 3, kh = warp >> 2, rho = 32 * q + lane;
     const int64_t n = block_row0 + rho;
     const float* const partial = reinterpret_cast<const float*>(smem_raw + SM::kWords);
+    const int col0 = kh * (NB / 2);
+    uint32_t w[NB / 2];
+    load_acc<NB / 2>(w, tmem_d + ((uint32_t)(q * 32) << 16) + col0, total > 0);
 #pragma unroll
-    for (int c0 = 0; c0 < NB / 2; c0 += 8) {
-      const int col = kh * (NB / 2) + c0;
-      uint32_t w[8];
-      load_acc8(w, tmem_d + ((uint32_t)(q * 32) << 16) + col, total > 0);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        float v = __uint_as_float(w[j]);
-        for (int r = 1; r < ksplit; ++r) v += partial[((r - 1) * NB + col + j) * kBM + rho];   // fixed order
-        if (col + j < M && n < N) y[(int64_t)(col + j) * N + n] = (uint16_t)float_to_bf16_bits(v);
-      }
+    for (int j = 0; j < NB / 2; ++j) {
+      float v = __uint_as_float(w[j]);
+      for (int r = 1; r < ksplit; ++r) v += partial[((r - 1) * NB + col0 + j) * kBM + rho];   // fixed order
+      if (col0 + j < M && n < N) y[(int64_t)(col0 + j) * N + n] = (uint16_t)float_to_bf16_bits(v);
     }
   }
   tc_fence_before_sync();
