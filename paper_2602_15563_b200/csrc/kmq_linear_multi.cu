@@ -20,8 +20,6 @@
 namespace kmq {
 namespace {
 
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
 constexpr int kTableBytesPerTile = 2 * 16 * 32 * 4;   // b = 4: [half][entry][lane] words
 constexpr int kMaxSmem = 200 * 1024;                  // dynamic shared memory a variant may ask for
 
@@ -36,11 +34,11 @@ struct MGeo {
   static constexpr int kPiecesPerRow = kStepK / 8;        // 16-byte pieces per batch row and step
 };
 
-// TPC tiles per CTA (2 or 4) -> 8 / TPC K-groups of TPC warps
-template <int BITS, int NT, int TPC>
+// TPC tiles per CTA (2 or 4), W warps -> W / TPC K-groups of TPC warps
+template <int BITS, int NT, int TPC, int W = 8>
 struct MSmem {
   using G = MGeo<BITS>;
-  static constexpr int kGroups = kWarps / TPC;
+  static constexpr int kGroups = W / TPC;
   static constexpr int kTableBytes = BITS == 4 ? TPC * kTableBytesPerTile : 0;
   static constexpr int kBuf = 8 * NT * G::kRowStride;                 // one x buffer: 8 NT batch rows of one step
   static constexpr int kX = kGroups * 2 * kBuf;                       // double buffered, per K-group
@@ -67,14 +65,15 @@ __device__ __forceinline__ void group_barrier(int group, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(group + 1), "r"(threads) : "memory");
 }
 
-template <int BITS, int NT, int TPC>
-__global__ void __launch_bounds__(kThreads, (NT <= 2 && TPC == 2) ? 2 : 1) linear_multi_kernel(const uint32_t* __restrict__ packed,
+template <int BITS, int NT, int TPC, int W = 8>
+__global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 1) linear_multi_kernel(const uint32_t* __restrict__ packed,
                                                                     const uint16_t* __restrict__ cb,
                                                                     const uint16_t* __restrict__ x,
                                                                     uint16_t* __restrict__ y, int64_t N, int64_t K,
                                                                     int M) {
   using G = MGeo<BITS>;
-  using SM = MSmem<BITS, NT, TPC>;
+  using SM = MSmem<BITS, NT, TPC, W>;
+  constexpr int kThreads = W * 32;
   constexpr int Q = G::kMmaPerWord;
   constexpr int kGroups = SM::kGroups, kGroupThreads = TPC * 32;
   constexpr int kSumRows = 8 * NT / TPC;   // b = 1: batch rows whose activations one warp sums
@@ -288,22 +287,22 @@ __global__ void __launch_bounds__(kThreads, (NT <= 2 && TPC == 2) ? 2 : 1) linea
   }
 }
 
-template <int BITS, int NT, int TPC>
+template <int BITS, int NT, int TPC, int W = 8>
 cudaError_t launch_nt(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N, int64_t K,
                       int M, cudaStream_t s) {
-  constexpr int smem = MSmem<BITS, NT, TPC>::kTotal;
+  constexpr int smem = MSmem<BITS, NT, TPC, W>::kTotal;
   static bool configured[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 64 && !configured[dev]) {
     cudaError_t e =
-        cudaFuncSetAttribute(linear_multi_kernel<BITS, NT, TPC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaFuncSetAttribute(linear_multi_kernel<BITS, NT, TPC, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   const int64_t tiles = (N + kTileRows - 1) / kTileRows;
   const unsigned grid = (unsigned)((tiles + TPC - 1) / TPC);
-  linear_multi_kernel<BITS, NT, TPC><<<grid, kThreads, smem, s>>>(packed, cb, x, y, N, K, M);
+  linear_multi_kernel<BITS, NT, TPC, W><<<grid, W * 32, smem, s>>>(packed, cb, x, y, N, K, M);
   return cudaGetLastError();
 }
 
@@ -315,17 +314,29 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
   const DeviceInfo* di = device_info();
   const int64_t tiles = (N + kTileRows - 1) / kTileRows;
   const bool few = (tiles + 3) / 4 <= (di ? di->sm_count : 148) / 2;
+  const bool fits_one_wave = (tiles + 3) / 4 <= (di ? di->sm_count : 148);   // CTAs of 4 tiles <= SMs
   if (M <= 8) {
+    // same shape of CTA for up to 8 batch rows (8192 x 28672, b = 1, M = 4: 35.0 -> 23.5 us; 8192 x 8192, b = 2,
+    // M = 8: 12.7 -> 11.7 us)
+    if (!few && fits_one_wave) return launch_nt<BITS, 1, 4, 16>(packed, cb, x, y, N, K, M, s);
     if (few || BITS != 1) return launch_nt<BITS, 1, 2>(packed, cb, x, y, N, K, M, s);
     return launch_nt<BITS, 1, 4>(packed, cb, x, y, N, K, M, s);
   }
   if (M <= 16) {
+    // 4 tiles x 4 K-groups (16 warps) when that grid gives every SM at most one CTA: 8192 x 8192, b = 2, M = 16:
+    // 16.1 -> 14.4 us; 8192 x 28672, M = 16: b = 1 47.9 -> 40.1 us, b = 4 85.2 -> 76.6 us
+    if (!few && fits_one_wave) return launch_nt<BITS, 2, 4, 16>(packed, cb, x, y, N, K, M, s);
     if (few || BITS != 1) return launch_nt<BITS, 2, 2>(packed, cb, x, y, N, K, M, s);
     return launch_nt<BITS, 2, 4>(packed, cb, x, y, N, K, M, s);
   }
   if (M <= 32) {
     if constexpr (MSmem<BITS, 4, 2>::kTotal <= kMaxSmem) {
       if (few) return launch_nt<BITS, 4, 2>(packed, cb, x, y, N, K, M, s);
+    }
+    // when every SM gets at most one CTA anyway: 4 K-groups, i.e. 16 warps per CTA instead of 8 (8192 x 8192,
+    // b = 2, M = 32: 22.6 -> 20.3 us; with more CTAs than SMs two 8-warp CTAs share an SM and that is faster)
+    if constexpr (MSmem<BITS, 4, 4, 16>::kTotal <= kMaxSmem) {
+      if (fits_one_wave) return launch_nt<BITS, 4, 4, 16>(packed, cb, x, y, N, K, M, s);
     }
     return launch_nt<BITS, 4, 4>(packed, cb, x, y, N, K, M, s);
   }
@@ -345,14 +356,16 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
 int linear_multi_rows_per_launch(int bits) { return bits == 1 ? 32 : 64; }
 
 // Smallest batch that goes to the multi-tile kernel.  The GEMV kernel stages the activations of a step once per
-// warp and tile; at b = 1 a step spans 512 activations per batch row against 1 KB of packed words, so from 4 batch
-// rows on sharing the staged activations among the tiles of a CTA wins (8192 x 28672, M = 8: 88 -> 37 us).  At
-// b = 2, 4 it only wins from 5 rows on and when the GEMV grid would not fit the SMs in one wave of CTAs.
+// warp and tile; at b = 1 a step spans 512 activations per batch row against 1 KB of packed words, so from 3 batch
+// rows on sharing the staged activations among the tiles of a CTA wins (8192 x 28672: 33 -> 23 us at M = 3,
+// 88 -> 25 us at M = 8), from 2 rows on when the GEMV grid would not fit the SMs in one wave of CTAs.  At b = 2, 4 it
+// only wins on such shapes, from 5 and 4 rows on.
 int linear_multi_min_rows(int bits, int64_t N) {
-  if (bits == 1) return 4;
   const DeviceInfo* di = device_info();
   const int64_t tiles = (N + kTileRows - 1) / kTileRows;
-  return (di && tiles > (int64_t)di->sm_count * 3) ? 5 : 9;
+  const bool waves = di && tiles > (int64_t)di->sm_count * 3;
+  if (bits == 1) return waves ? 2 : 3;
+  return waves ? (bits == 2 ? 5 : 4) : 9;
 }
 
 cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
