@@ -315,10 +315,16 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
   const int64_t tiles = (N + kTileRows - 1) / kTileRows;
   const bool few = (tiles + 3) / 4 <= (di ? di->sm_count : 148) / 2;
   const bool fits_one_wave = (tiles + 3) / 4 <= (di ? di->sm_count : 148);   // CTAs of 4 tiles <= SMs
+  // few tiles and a long K: 2 tiles x 8 K-groups (16 warps) while each K-group still gets 4 steps or more
+  // (4096 x 11008, b = 2, M = 16: 13.4 -> 12.3 us; 4096 x 4096: b = 4 11.5 -> 9.8 us, b = 2 (16 steps) 6.4 -> 6.9 us)
+  const bool few16 = few && (tiles + 1) / 2 <= (di ? di->sm_count : 148) && (K * BITS / 128 + 3) / 4 >= 32;
   if (M <= 8) {
     // same shape of CTA for up to 8 batch rows (8192 x 28672, b = 1, M = 4: 35.0 -> 23.5 us; 8192 x 8192, b = 2,
     // M = 8: 12.7 -> 11.7 us)
     if (!few && fits_one_wave) return launch_nt<BITS, 1, 4, 16>(packed, cb, x, y, N, K, M, s);
+    if constexpr (MSmem<BITS, 1, 2, 16>::kTotal <= kMaxSmem) {
+      if (few16) return launch_nt<BITS, 1, 2, 16>(packed, cb, x, y, N, K, M, s);
+    }
     if (few || BITS != 1) return launch_nt<BITS, 1, 2>(packed, cb, x, y, N, K, M, s);
     return launch_nt<BITS, 1, 4>(packed, cb, x, y, N, K, M, s);
   }
@@ -326,6 +332,9 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
     // 4 tiles x 4 K-groups (16 warps) when that grid gives every SM at most one CTA: 8192 x 8192, b = 2, M = 16:
     // 16.1 -> 14.4 us; 8192 x 28672, M = 16: b = 1 47.9 -> 40.1 us, b = 4 85.2 -> 76.6 us
     if (!few && fits_one_wave) return launch_nt<BITS, 2, 4, 16>(packed, cb, x, y, N, K, M, s);
+    if constexpr (MSmem<BITS, 2, 2, 16>::kTotal <= kMaxSmem) {
+      if (few16) return launch_nt<BITS, 2, 2, 16>(packed, cb, x, y, N, K, M, s);
+    }
     if (few || BITS != 1) return launch_nt<BITS, 2, 2>(packed, cb, x, y, N, K, M, s);
     return launch_nt<BITS, 2, 4>(packed, cb, x, y, N, K, M, s);
   }
