@@ -275,8 +275,10 @@ def run_library(args):
         barrier()
         sampler.active = False
     elapsed_ms = t0.elapsed_time(t1)
-    per_case_ms = [sum(ev[s][j][0].elapsed_time(ev[s][j][1]) for s in range(args.steps)) / args.steps
-                   for j in range(len(cases))]
+    step_ms = [[ev[s][j][0].elapsed_time(ev[s][j][1]) for s in range(args.steps)] for j in range(len(cases))]
+    per_case_ms = [sum(t) / args.steps for t in step_ms]
+    # standard error of the mean per-call time over the K timed steps (each step = one replay of the case's graph)
+    per_case_sem_ms = [(float(np.std(t, ddof=1)) / np.sqrt(len(t)) if len(t) > 1 else 0.0) for t in step_ms]
 
     step_bytes = sum(c.bytes * c.pool for c in cases)
     step_calls = sum(c.pool for c in cases)
@@ -348,11 +350,12 @@ def run_library(args):
 
     # ---- per-case figures and the roofline of the dominant kernel ----
     per_case = []
-    for c, ms in zip(cases, per_case_ms):
+    for c, ms, sem in zip(cases, per_case_ms, per_case_sem_ms):
         us = ms * 1e3 / c.pool
         gbs = c.bytes / (us * 1e-6) / 1e9
         per_case.append({"layer": c.name, "N": c.N, "K": c.K, "bits": c.bits, "M": c.M, "pool": c.pool,
-                         "variant": c.variant, "us_per_call": round(us, 3), "gbs": round(gbs, 1),
+                         "variant": c.variant, "us_per_call": round(us, 3),
+                         "us_per_call_sem": round(sem * 1e3 / c.pool, 4), "gbs": round(gbs, 1),
                          "frac_of_measured_hbm": round(gbs / peak_gbs, 4), "frac_of_8tbs": round(gbs / 8000.0, 4),
                          "bytes_per_call": c.bytes})
     dom = max(range(len(cases)), key=lambda j: per_case_ms[j])
@@ -386,6 +389,7 @@ def run_library(args):
         "gpu_launches": args.steps * sum(c.pool * c.launches for c in cases),
         "clocks": sampler.summary(),
         "parity": {"calls_checked": checked, "max_err_over_tol": round(worst, 4), "ok": bool(worst <= 1.0)},
+        "paper_context": PAPER_CONTEXT,
     }
     print(json.dumps(line))
     if dist is not None:
@@ -395,6 +399,17 @@ def run_library(args):
 # --------------------------------------------------------------------------
 # the CPU oracle, timed (reported baseline and the reference arm)
 # --------------------------------------------------------------------------
+# The paper's own kernel timings (Appendix "Benchmarking", table of the 1 x 8192 by 8192 x 8192 product at batch 1).
+# Other hardware and another format: context only, not a target and not comparable row by row.
+PAPER_CONTEXT = {
+    "note": "paper's numbers: one NVIDIA L40S (864 GB/s), shared 256-entry byte LUT + bf16 block scales (B = 64), "
+            "Triton kernels, 8192 x 8192 at batch 1; context only",
+    "bf16_16bit": {"us": 175.6, "gbs": 764, "frac_of_l40s_peak": 0.88},
+    "kmeans_4p25bit": {"us": 49.5, "gbs": 721, "frac_of_l40s_peak": 0.83},
+    "kmeans_1p25bit": {"us": 24.0, "gbs": 438, "frac_of_l40s_peak": 0.51},
+}
+
+
 def _cpu_threads():
     try:
         from threadpoolctl import threadpool_info
