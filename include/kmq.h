@@ -175,11 +175,11 @@ size_t kmq_static_scratch_capacity(void);
  * 128 output rows are dequantised straight into tensor memory as the A
  * operand of tcgen05.mma, the activations are the B operand in shared
  * memory, the accumulator lives in tensor memory.  `packed` must be in
- * KMQ_LAYOUT_TUNED and K * bits a multiple of 128; any M >= 1 (64 batch rows
+ * KMQ_LAYOUT_TUNED and K * bits a multiple of 128; any M >= 1 (128 batch rows
  * per launch).  This is the large-batch design the paper's roofline model
  * points to (Appendix "Theoretical model": beyond a batch of P_w * nu / 16
  * the layer is compute bound).  One tcgen05.mma (2048 weights) costs 70 to
- * 100 clocks whatever the batch, so the time does not depend on M up to 64
+ * 100 clocks whatever the batch, so the time does not depend on M up to 128
  * rows but a CTA covers 128 output rows: kmq_linear itself selects this
  * kernel for M > 32 on shapes with enough 128-row blocks to occupy most SMs
  * (kmq_linear_variant() then starts with "tcgen05"); this entry point forces

@@ -41,11 +41,13 @@ constexpr int kBM = 128;                                 // output rows per CTA 
 constexpr int kDecodeWarps = 16;                         // 4 tensor-memory lane quarters x 4 quarters of a stage's weights
 constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kThreads = kDecodeThreads + 64;            // + the MMA warp + the TMA producer warp
-#ifndef KMQ_UMMA_ARING
-#define KMQ_UMMA_ARING 6
-#endif
-constexpr int kARing = KMQ_UMMA_ARING;                   // A operands in tensor memory: the decoders may run this far ahead
-constexpr int kBRing = kARing;                           // B buffers in shared memory, one per A operand
+// Stages in flight: A operands in tensor memory (the decoders may run this far ahead of the MMAs) and, one per A
+// operand, B buffers in shared memory.  6, or 4 for more than 64 batch rows (128 columns of accumulator, 32 KB per B
+// buffer).
+template <int NB>
+constexpr int ring_depth() {
+  return NB > 64 ? 4 : 6;
+}
 #ifndef KMQ_UMMA_WRING
 #define KMQ_UMMA_WRING 6
 #endif
@@ -62,13 +64,15 @@ struct UGeo {
   static constexpr int kThreadBytes = kStageK * BITS / 32;       // packed bytes a thread decodes per stage: 16, 8, 4
   static constexpr int kCols = kStageK / 2;                      // 32-bit columns of the A operand of a stage
   static constexpr int kKSlices = kStageK / 16;                  // MMAs per stage
-  static constexpr int kTmemCols = kARing * 64 + 64 <= 256 ? 256 : 512;   // kARing * kCols + up to 64 columns of D, a power of two
-  static_assert(kARing * 64 + 64 <= 512, "tensor memory has 512 columns");
   static constexpr int kTableBytes = BITS == 4 ? 4 * 16 * 128 : 0;   // b = 4: [lane quarter][entry][lane]
 };
 
 template <int BITS, int NB>
 struct USmem {
+  static constexpr int kARing = ring_depth<NB>();
+  static constexpr int kBRing = kARing;
+  static constexpr int kTmemCols = 512;                             // kARing * 64 columns of A + NB columns of D <= 512
+  static_assert(kARing * 64 + NB <= 512, "tensor memory has 512 columns");
   static constexpr int kBHalfBytes = NB * 128;                      // NB rows x 64 activations (one TMA box)
   static constexpr int kBStageBytes = 2 * kBHalfBytes;
   static constexpr int kB = 0;
@@ -268,6 +272,9 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
   using SM = USmem<BITS, NB>;
   constexpr int SPS = G::kStagesPerStep;
   constexpr int NW = G::kThreadBytes / 4;   // packed words per thread and stage: 4, 2, 1
+  constexpr int kARing = SM::kARing;
+  constexpr int kReaders = NB % 32 == 0 ? 4 : 2;   // warps per lane quarter that read the accumulator
+  constexpr int kReadCols = NB / kReaders;         // columns each of them reads (a multiple of 8)
   extern __shared__ __align__(1024) unsigned char smem_unaligned[];
   unsigned char* const smem_raw =
       smem_unaligned + ((1024u - ((uint32_t)__cvta_generic_to_shared(smem_unaligned) & 1023u)) & 1023u);
@@ -300,7 +307,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
   }
   if (warp == kDecodeWarps) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_base + SM::kTmemSlot),
-                 "r"((uint32_t)G::kTmemCols)
+                 "r"((uint32_t)SM::kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -454,21 +461,21 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
     if (!ok) atomicOr(&g_device_error_flags, 1u);
   }
   // ---- accumulators of the cluster -> rank 0 -> bf16 ----
-  // Rank r > 0 hands its accumulator to rank 0 through rank 0's shared memory (the ring of packed words, free once
-  // every CTA of the cluster has left its main loop): [r - 1][batch row][output row] floats.
+  // Rank r > 0 hands its accumulator to rank 0 through rank 0's shared memory (the B buffers, free once every CTA of
+  // the cluster has seen its last MMA complete): [r - 1][batch row][output row] floats.
   __syncwarp();
   if (ksplit > 1) cluster_sync();
-  const bool reader = warp < kDecodeWarps && (warp >> 2) < 2 && ok;   // two warps per lane quarter split the columns
+  const bool reader = warp < kDecodeWarps && (warp >> 2) < kReaders && ok;   // the warps of a lane quarter split the columns
   if (reader) {
     const int q = warp & 3, kh = warp >> 2, rho = 32 * q + lane;
     tc_fence_after_sync();
     if (rank != 0) {
-      const uint32_t remote = map_to_rank0(smem_base + SM::kWords) + (uint32_t)(rank - 1) * (NB * kBM * 4);
-      const int col0 = kh * (NB / 2);
-      uint32_t w[NB / 2];
-      load_acc<NB / 2>(w, tmem_d + ((uint32_t)(q * 32) << 16) + col0, total > 0);
+      const uint32_t remote = map_to_rank0(smem_base + SM::kB) + (uint32_t)(rank - 1) * (NB * kBM * 4);
+      const int col0 = kh * kReadCols;
+      uint32_t w[kReadCols];
+      load_acc<kReadCols>(w, tmem_d + ((uint32_t)(q * 32) << 16) + col0, total > 0);
 #pragma unroll
-      for (int j = 0; j < NB / 2; ++j)
+      for (int j = 0; j < kReadCols; ++j)
         asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(remote + ((col0 + j) * kBM + rho) * 4), "r"(w[j]) : "memory");
     }
   }
@@ -477,12 +484,12 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
   if (reader && rank == 0) {
     const int q = warp & 3, kh = warp >> 2, rho = 32 * q + lane;
     const int64_t n = block_row0 + rho;
-    const float* const partial = reinterpret_cast<const float*>(smem_raw + SM::kWords);
-    const int col0 = kh * (NB / 2);
-    uint32_t w[NB / 2];
-    load_acc<NB / 2>(w, tmem_d + ((uint32_t)(q * 32) << 16) + col0, total > 0);
+    const float* const partial = reinterpret_cast<const float*>(smem_raw + SM::kB);
+    const int col0 = kh * kReadCols;
+    uint32_t w[kReadCols];
+    load_acc<kReadCols>(w, tmem_d + ((uint32_t)(q * 32) << 16) + col0, total > 0);
 #pragma unroll
-    for (int j = 0; j < NB / 2; ++j) {
+    for (int j = 0; j < kReadCols; ++j) {
       float v = __uint_as_float(w[j]);
       for (int r = 1; r < ksplit; ++r) v += partial[((r - 1) * NB + col0 + j) * kBM + rho];   // fixed order
       if (col0 + j < M && n < N) y[(int64_t)(col0 + j) * N + n] = (uint16_t)float_to_bf16_bits(v);
@@ -491,7 +498,7 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
   tc_fence_before_sync();
   __syncthreads();
   if (warp == kDecodeWarps)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)G::kTmemCols)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)SM::kTmemCols)
                  : "memory");
 }
 
@@ -543,7 +550,8 @@ cudaError_t launch_nb(const uint32_t* packed, const uint16_t* cb, const uint16_t
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  static_assert(NB * kBM * 4 <= kWRing * kWStepBytes, "the partial accumulator of the second CTA must fit the words ring");
+  static_assert(NB * kBM * 4 <= USmem<BITS, NB>::kBRing * USmem<BITS, NB>::kBStageBytes,
+                "the partial accumulator of the second CTA must fit the B buffers");
   CUtensorMap xmap;
   if (!make_x_map<NB>(&xmap, x, K, M)) return cudaErrorInvalidValue;
   const unsigned blocks = (unsigned)((N + kBM - 1) / kBM);
@@ -569,12 +577,14 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
   if (M <= 16) return launch_nb<BITS, 16>(packed, cb, x, y, N, K, M, s);
   if (M <= 32) return launch_nb<BITS, 32>(packed, cb, x, y, N, K, M, s);
   if (M <= 48) return launch_nb<BITS, 48>(packed, cb, x, y, N, K, M, s);
-  return launch_nb<BITS, 64>(packed, cb, x, y, N, K, M, s);
+  if (M <= 64) return launch_nb<BITS, 64>(packed, cb, x, y, N, K, M, s);
+  if (M <= 96) return launch_nb<BITS, 96>(packed, cb, x, y, N, K, M, s);
+  return launch_nb<BITS, 128>(packed, cb, x, y, N, K, M, s);
 }
 
 }  // namespace
 
-int linear_umma_rows_per_launch() { return 64; }
+int linear_umma_rows_per_launch() { return 128; }   // one tcgen05.mma costs the same for every N <= 128
 
 // CTAs per 128-row block: K is split over a cluster of 2 (partial sums meet in CTA 0's shared memory) while the
 // blocks alone would leave at least half of the SMs idle and each half still has a few steps.
@@ -585,13 +595,14 @@ int linear_umma_ksplit(int64_t N, int64_t K, int bits) {
 }
 
 // The tensor core issues one tcgen05.mma (2048 weights) per 70-100 clocks whatever the batch, so the kernel's time
-// does not depend on M up to 64 rows, but a CTA covers 128 output rows: it pays when the batch is large and there
+// does not depend on M up to 128 rows, but a CTA covers 128 output rows: it pays when the batch is large and there
 // are enough 128-row blocks to occupy most SMs.  Measured: 16384 x 3072, b = 2: 18.5 us for any M <= 64 against
 // 18.5 / 28.5 / 31.6 us of the multi-tile kernel at M = 32 / 40 / 64; 12288 x 4096, M = 64: 22.7 against 38.9 us;
 // 8192 x 8192 (64 blocks), M = 64: 38.9 against 36.0 us.
 bool linear_umma_selected(int64_t N, int64_t K, int bits, int64_t M) {
   const DeviceInfo* di = device_info();
   if (!di || M <= 32 || (K * bits) % 128 != 0) return false;
+  if (!encode_tiled()) return false;   // no tensor-map encoder in this driver: stay on the mma.sync kernels
   return (N + kBM - 1) / kBM * linear_umma_ksplit(N, K, bits) >= (int64_t)di->sm_count * 5 / 8;
 }
 

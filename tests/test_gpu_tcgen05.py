@@ -36,7 +36,8 @@ def run(idx, cb, x, bits):
 # ragged row counts (not a multiple of 16 or 128), K that is not a whole number of stages, every width of the MMA's N
 @pytest.mark.parametrize("bits", (1, 2, 4))
 @pytest.mark.parametrize("N,Kmul,M", [(128, 4, 16), (200, 9, 48), (333, 5, 64), (77, 12, 17), (1000, 32, 33),
-                                      (129, 2, 31), (16, 1, 1), (48, 1, 64), (520, 16, 130), (2048, 64, 20)])
+                                      (129, 2, 31), (16, 1, 1), (48, 1, 64), (520, 16, 130), (2048, 64, 20), (300, 8, 90),
+                                      (1100, 32, 128)])
 def test_tcgen05_linear_matches_oracle(bits, N, Kmul, M):
     K = (128 // bits) * Kmul          # Kmul 16-byte chunks per row
     rng = np.random.default_rng(9000 + 100 * bits + N + M)
