@@ -550,12 +550,12 @@ cudaError_t launch_nb(const uint32_t* packed, const uint16_t* cb, const uint16_t
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  static_assert(NB * kBM * 4 <= USmem<BITS, NB>::kBRing * USmem<BITS, NB>::kBStageBytes,
-                "the partial accumulator of the second CTA must fit the B buffers");
   CUtensorMap xmap;
   if (!make_x_map<NB>(&xmap, x, K, M)) return cudaErrorInvalidValue;
   const unsigned blocks = (unsigned)((N + kBM - 1) / kBM);
-  const int ksplit = linear_umma_ksplit(N, K, BITS);
+  const int ksplit = linear_umma_ksplit(N, K, BITS, NB);
+  if ((ksplit - 1) * NB * kBM * 4 > USmem<BITS, NB>::kBRing * USmem<BITS, NB>::kBStageBytes)
+    return cudaErrorInvalidValue;   // the partial accumulators of the other CTAs must fit the B buffers
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(blocks, (unsigned)ksplit);
   cfg.blockDim = dim3(kThreads);
@@ -586,12 +586,15 @@ cudaError_t launch_bits(const uint32_t* packed, const uint16_t* cb, const uint16
 
 int linear_umma_rows_per_launch() { return 128; }   // one tcgen05.mma costs the same for every N <= 128
 
-// CTAs per 128-row block: K is split over a cluster of 2 (partial sums meet in CTA 0's shared memory) while the
-// blocks alone would leave at least half of the SMs idle and each half still has a few steps.
-int linear_umma_ksplit(int64_t N, int64_t K, int bits) {
+// CTAs per 128-row block: K is split over a cluster of 2 or 4 (partial sums meet in CTA 0's shared memory) while the
+// blocks alone would leave at least half (three quarters) of the SMs idle and each part still has a few steps.
+// `batch` = rows of one launch; 4 CTAs only up to 64 rows (three partial accumulators must fit the B buffers).
+int linear_umma_ksplit(int64_t N, int64_t K, int bits, int batch) {
   const DeviceInfo* di = device_info();
+  if (!di) return 1;
   const int64_t blocks = (N + kBM - 1) / kBM, steps = (K * bits / 128 + 3) / 4;
-  return (di && blocks * 2 <= di->sm_count && steps >= 8) ? 2 : 1;
+  if (blocks * 4 <= di->sm_count && steps >= 32 && batch <= 64) return 4;   // measured: no gain with fewer than 8 steps per CTA
+  return (blocks * 2 <= di->sm_count && steps >= 8) ? 2 : 1;
 }
 
 // The tensor core issues one tcgen05.mma (2048 weights) per 70-100 clocks whatever the batch, so the kernel's time
@@ -603,7 +606,12 @@ bool linear_umma_selected(int64_t N, int64_t K, int bits, int64_t M) {
   const DeviceInfo* di = device_info();
   if (!di || M <= 32 || (K * bits) % 128 != 0) return false;
   if (!encode_tiled()) return false;   // no tensor-map encoder in this driver: stay on the mma.sync kernels
-  return (N + kBM - 1) / kBM * linear_umma_ksplit(N, K, bits) >= (int64_t)di->sm_count * 5 / 8;
+  const int batch = (int)(M < linear_umma_rows_per_launch() ? M : linear_umma_rows_per_launch());
+  const int64_t ctas = (N + kBM - 1) / kBM * linear_umma_ksplit(N, K, bits, batch);
+  // with fewer CTAs it still wins where the multi-tile kernel is weakest: more than 48 rows, or b = 1 (which that
+  // kernel serves 32 rows at a time): 4096 x 4096, 64 CTAs, M = 64: b = 2 18.4 against 20.7 us, b = 1 17.6 against 32.8 us
+  const int64_t need = (M > 48 || bits == 1) ? (int64_t)di->sm_count * 3 / 8 : (int64_t)di->sm_count * 5 / 8;
+  return ctas >= need;
 }
 
 cudaError_t launch_linear_umma(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,

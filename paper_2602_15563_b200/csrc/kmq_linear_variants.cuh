@@ -34,7 +34,7 @@ cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, cons
                                 int64_t K, int bits, int64_t M, cudaStream_t s);
 bool linear_umma_selected(int64_t N, int64_t K, int bits, int64_t M);   // kmq_linear's choice of the tcgen05 kernel
 int linear_umma_rows_per_launch();
-int linear_umma_ksplit(int64_t N, int64_t K, int bits);   // CTAs (cluster size) per 128-row block
+int linear_umma_ksplit(int64_t N, int64_t K, int bits, int batch);   // CTAs (cluster size) per 128-row block
 cudaError_t launch_linear_umma(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                int64_t K, int bits, int64_t M, cudaStream_t s);
 cudaError_t read_device_error_flags(unsigned int* flags);   // synchronises; reads and clears the sticky error word
