@@ -37,7 +37,8 @@ def run(idx, cb, x, bits):
 @pytest.mark.parametrize("bits", (1, 2, 4))
 @pytest.mark.parametrize("N,Kmul,M", [(128, 4, 16), (200, 9, 48), (333, 5, 64), (77, 12, 17), (1000, 32, 33),
                                       (129, 2, 31), (16, 1, 1), (48, 1, 64), (520, 16, 130), (2048, 64, 20), (300, 8, 90),
-                                      (1100, 32, 128)])
+                                      (1100, 32, 128),
+                                      (520, 128, 64), (300, 131, 33)])   # >= 32 steps of K: cluster of 4 CTAs
 def test_tcgen05_linear_matches_oracle(bits, N, Kmul, M):
     K = (128 // bits) * Kmul          # Kmul 16-byte chunks per row
     rng = np.random.default_rng(9000 + 100 * bits + N + M)
