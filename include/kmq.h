@@ -181,7 +181,7 @@ size_t kmq_static_scratch_capacity(void);
  * the layer is compute bound).  One tcgen05.mma (2048 weights) costs 70 to
  * 100 clocks whatever the batch, so the time does not depend on M up to 128
  * rows but a CTA covers 128 output rows: kmq_linear itself selects this
- * kernel for M > 32 on shapes with enough 128-row blocks to occupy most SMs
+ * kernel for M > 32 (b = 1: M > 16) on shapes with enough 128-row blocks to occupy most SMs
  * (kmq_linear_variant() then starts with "tcgen05"); this entry point forces
  * it for any shape.
  * It needs no workspace.  Its waits on hardware barriers are bounded, see

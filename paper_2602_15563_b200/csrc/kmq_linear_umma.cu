@@ -604,7 +604,9 @@ int linear_umma_ksplit(int64_t N, int64_t K, int bits, int batch) {
 // 8192 x 8192 (64 blocks), M = 64: 38.9 against 36.0 us.
 bool linear_umma_selected(int64_t N, int64_t K, int bits, int64_t M) {
   const DeviceInfo* di = device_info();
-  if (!di || M <= 32 || (K * bits) % 128 != 0) return false;
+  // b = 1: the multi-tile kernel has no 16-warp form beyond 16 rows (its x buffers are twice as large) and takes
+  // 80 us at 8192 x 28672 for M = 17..32 against 60 us here
+  if (!di || M <= (bits == 1 ? 16 : 32) || (K * bits) % 128 != 0) return false;
   if (!encode_tiled()) return false;   // no tensor-map encoder in this driver: stay on the mma.sync kernels
   const int batch = (int)(M < linear_umma_rows_per_launch() ? M : linear_umma_rows_per_launch());
   const int64_t ctas = (N + kBM - 1) / kBM * linear_umma_ksplit(N, K, bits, batch);
