@@ -19,7 +19,7 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
       p.name = bits == 4 ? "tcgen05_table_b4" : bits == 2 ? "tcgen05_prmt_b2" : "tcgen05_select_b1";
       return p;
     }
-    if (tuned && M >= linear_multi_min_rows(bits, N, K)) {
+    if (tuned && M >= linear_multi_min_rows(bits, N)) {
       const int64_t per = linear_multi_rows_per_launch(bits);
       p.variant = kVariantMulti;
       p.launches = (int)((M + per - 1) / per);

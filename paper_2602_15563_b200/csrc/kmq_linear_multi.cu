@@ -368,17 +368,13 @@ int linear_multi_rows_per_launch(int bits) { return bits == 1 ? 32 : 64; }
 // warp and tile; at b = 1 a step spans 512 activations per batch row against 1 KB of packed words, so from 3 batch
 // rows on sharing the staged activations among the tiles of a CTA wins (8192 x 28672: 33 -> 23 us at M = 3,
 // 88 -> 25 us at M = 8), from 2 rows on when the GEMV grid would not fit the SMs in one wave of CTAs.  At b = 2, 4 it
-// only wins on such shapes, from 5 and 4 rows on -- at b = 2 from 2 rows on when K is long and the 16-warp CTAs apply
-// (8192 x 8192: 11.2 against 12.1 us at M = 2, 11.3 against 12.6 us at M = 4; 8192 x 4096: 6.9 against 6.7 us).
-int linear_multi_min_rows(int bits, int64_t N, int64_t K) {
+// only wins on such shapes, from 5 and 4 rows on.
+int linear_multi_min_rows(int bits, int64_t N) {
   const DeviceInfo* di = device_info();
   const int64_t tiles = (N + kTileRows - 1) / kTileRows;
   const bool waves = di && tiles > (int64_t)di->sm_count * 3;
   if (bits == 1) return waves ? 2 : 3;
-  if (!waves) return 9;
-  if (bits == 4) return 4;
-  const bool one_cta_per_sm = (tiles + 3) / 4 <= di->sm_count;
-  return (one_cta_per_sm && (K * bits / 128 + 3) / 4 >= 32) ? 2 : 5;
+  return waves ? (bits == 2 ? 5 : 4) : 9;
 }
 
 cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
@@ -389,7 +385,7 @@ cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, cons
     const uint16_t* xp = x + m0 * K;
     uint16_t* yp = y + m0 * N;
     cudaError_t e;
-    if (mc < linear_multi_min_rows(bits, N, K)) e = launch_linear_tiled(packed, cb, xp, yp, N, K, bits, mc, s);   // a short tail
+    if (mc < linear_multi_min_rows(bits, N)) e = launch_linear_tiled(packed, cb, xp, yp, N, K, bits, mc, s);   // a short tail
     else if (bits == 1) e = launch_bits<1>(packed, cb, xp, yp, N, K, mc, s);
     else if (bits == 2) e = launch_bits<2>(packed, cb, xp, yp, N, K, mc, s);
     else e = launch_bits<4>(packed, cb, xp, yp, N, K, mc, s);

@@ -489,7 +489,7 @@ constexpr int64_t kSplitMinSteps = KMQ_SPLIT_MIN_STEPS;
 
 int linear_split_ctas(int64_t N, int64_t K, int bits, int64_t M) {
   const DeviceInfo* di = device_info();
-  if (!di || M >= linear_multi_min_rows(bits, N, K)) return 0;
+  if (!di || M >= linear_multi_min_rows(bits, N)) return 0;
   const int64_t slots = (int64_t)di->sm_count * 3;
   const int64_t tiles = (N + kRows - 1) / kRows;
   const int64_t steps = (K * bits / 128 + 3) / 4;

@@ -29,7 +29,7 @@ size_t linear_split_scratch_bytes(int ctas);
 cudaError_t launch_linear_split(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                 int64_t K, int bits, int64_t M, void* scratch, int ctas, cudaStream_t s);
 int linear_multi_rows_per_launch(int bits);
-int linear_multi_min_rows(int bits, int64_t N, int64_t K);   // smallest batch routed to the multi-tile kernel
+int linear_multi_min_rows(int bits, int64_t N);   // smallest batch routed to the multi-tile kernel
 cudaError_t launch_linear_multi(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                 int64_t K, int bits, int64_t M, cudaStream_t s);
 bool linear_umma_selected(int64_t N, int64_t K, int bits, int64_t M);   // kmq_linear's choice of the tcgen05 kernel

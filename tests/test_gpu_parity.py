@@ -171,8 +171,8 @@ def test_workspace_is_checked_on_the_host():
 @pytest.mark.parametrize("Kmul,M", [(512, 1), (517, 3)])
 def test_linear_balanced_split_variant(bits, Kmul, M):
     N, K = 16 * 460 + 5, (128 // bits) * Kmul          # 461 tiles (the last one ragged), Kmul 16-byte chunks per row
-    if bits in (1, 2):
-        M = 1                                          # b = 1, 2 go to the multi-tile kernel from 2 batch rows on here
+    if bits == 1:
+        M = 1                                          # b = 1 goes to the multi-tile kernel from 2 batch rows on here
     rng = np.random.default_rng(7000 + 10 * bits + Kmul)
     idx, cb, x = random_layer(rng, N, K, bits, M)
     T = kmq.KMQ_LAYOUT_TUNED
