@@ -93,8 +93,11 @@ int kmq_packed_field_shift(int i, int bits, int layout);
  * (fp32 partial sums of a split along K); may be 0. */
 size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M, int layout);
 
-/* Number of kernels one kmq_linear call launches for this shape (1 or 2), and
- * a short static name of the kernel variant the dispatcher picks. */
+/* Number of kernels one kmq_linear call launches for this shape (one per pass
+ * of batch rows; 2 for the balanced split with its fix-up kernel), and a short
+ * static name of the kernel variant the dispatcher picks: "tiled_*", "split_*",
+ * "multi_*", "tcgen05_*" (tuned layout), "staged_*" (canonical layout),
+ * "generic_warp_per_row", or "invalid". */
 int kmq_linear_num_launches(int64_t N, int64_t K, int bits, int64_t M, int layout);
 const char* kmq_linear_variant(int64_t N, int64_t K, int bits, int64_t M, int layout);
 
@@ -181,7 +184,8 @@ size_t kmq_static_scratch_capacity(void);
  * the layer is compute bound).  One tcgen05.mma (2048 weights) costs 70 to
  * 100 clocks whatever the batch, so the time does not depend on M up to 128
  * rows but a CTA covers 128 output rows: kmq_linear itself selects this
- * kernel for M > 32 (b = 1: M > 16) on shapes with enough 128-row blocks to occupy most SMs
+ * kernel for M > 32 (b = 1: M > 16) on shapes with enough 128-row blocks to
+ * occupy most SMs
  * (kmq_linear_variant() then starts with "tcgen05"); this entry point forces
  * it for any shape.
  * It needs no workspace.  Its waits on hardware barriers are bounded, see
