@@ -84,6 +84,19 @@ def cached_layer(synth, N, K, bits, dist, config_id):
     return _LAYER_CACHE[key]
 
 
+def select_cases(args):
+    """The cases of the workload, or the subset named by --case (e.g. "bits=1,M=1" or "layer=qkv")."""
+    cases = WORKLOADS[args.workload]
+    if not args.case:
+        return cases
+    want = dict(kv.split("=") for kv in args.case.split(","))
+    keep = [c for c in cases if all(str({"layer": c[0], "N": c[1], "K": c[2], "bits": c[4], "M": c[5]}[k]) == v
+                                    for k, v in want.items())]
+    if not keep:
+        raise SystemExit(f"--case {args.case!r} matches no case of {args.workload}")
+    return keep
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -151,7 +164,7 @@ class ClockSampler(threading.Thread):
 class Case:
     """One (layer, bits, M) of the workload with its pool of device buffers."""
 
-    def __init__(self, name, N, K, dist, bits, M, config_id, torch, kmq, synth, pool_bytes):
+    def __init__(self, name, N, K, dist, bits, M, config_id, torch, kmq, synth, pool_bytes, layout="auto"):
         self.name, self.N, self.K, self.bits, self.M = name, N, K, bits, M
         self.bytes = algorithmic_bytes(N, K, bits, M)
         self.pool = max(4, -(-pool_bytes // self.bytes))
@@ -162,7 +175,13 @@ class Case:
         self.layer = layer
         dev = torch.device("cuda")
         idx = torch.from_numpy(layer["idx"]).to(dev)
-        self.layout = kmq.KMQ_LAYOUT_TUNED                         # the layout the fast kernels read
+        # the layout in which the library is fastest for this batch (packing is the offline step)
+        self.layout = {"tuned": kmq.KMQ_LAYOUT_TUNED, "table": kmq.KMQ_LAYOUT_TABLE,
+                       "canonical": kmq.KMQ_LAYOUT_CANONICAL}.get(layout)
+        if self.layout is None:
+            self.layout = kmq.kmq_preferred_layout(N, K, bits, M) if M > 0 else kmq.KMQ_LAYOUT_TUNED
+        self.layout_name = {kmq.KMQ_LAYOUT_TUNED: "tuned", kmq.KMQ_LAYOUT_TABLE: "table",
+                            kmq.KMQ_LAYOUT_CANONICAL: "canonical"}[self.layout]
         words = kmq.kmq_packed_bytes(N, K, bits, self.layout) // 4
         if self.dequant:
             self.pool = max(2, -(-pool_bytes // self.bytes))
@@ -226,8 +245,8 @@ def run_library(args):
     peak_gbs, peak_kind = measured_peak()
     cfg_id = CONFIG_ID[args.workload]
     pool_bytes = 2 * L2_BYTES
-    cases = [Case(n, N, K, d, b, M, cfg_id, torch, kmq, synth, pool_bytes)
-             for (n, N, K, d, b, M) in WORKLOADS[args.workload]]
+    cases = [Case(n, N, K, d, b, M, cfg_id, torch, kmq, synth, pool_bytes, args.layout)
+             for (n, N, K, d, b, M) in select_cases(args)]
 
     stream = torch.cuda.Stream()
     graphs = []
@@ -294,7 +313,7 @@ def run_library(args):
         sampler.stop_flag = True
         if rank == 0:
             for c, ms in zip(cases, per_case_ms):
-                print(f"{c.name} b={c.bits} M={c.M} [{c.variant}]: {ms * 1e3 / c.pool:.3f} us/call, "
+                print(f"{c.name} b={c.bits} M={c.M} [{c.variant}, {c.layout_name}]: {ms * 1e3 / c.pool:.3f} us/call, "
                       f"{c.bytes / (ms * 1e-3 / c.pool) / 1e9:.1f} GB/s")
         if dist is not None:
             dist.destroy_process_group()
@@ -354,7 +373,7 @@ def run_library(args):
         us = ms * 1e3 / c.pool
         gbs = c.bytes / (us * 1e-6) / 1e9
         per_case.append({"layer": c.name, "N": c.N, "K": c.K, "bits": c.bits, "M": c.M, "pool": c.pool,
-                         "variant": c.variant, "us_per_call": round(us, 3),
+                         "variant": c.variant, "layout": c.layout_name, "us_per_call": round(us, 3),
                          "us_per_call_sem": round(sem * 1e3 / c.pool, 4), "gbs": round(gbs, 1),
                          "frac_of_measured_hbm": round(gbs / peak_gbs, 4), "frac_of_8tbs": round(gbs / 8000.0, 4),
                          "bytes_per_call": c.bytes})
@@ -378,7 +397,8 @@ def run_library(args):
                    "calls_per_step": step_calls, "bytes_per_step": step_bytes,
                    "l2": "inputs larger than L2: every call of a step uses its own weight set, pool >= 2 x 126 MB",
                    "launch": "CUDA graph per case, replayed once per step", "multi_gpu": "replicas only",
-                   "packed_layout": "tuned (tile-major), packed once by kmq_pack before the timed region"},
+                   "packed_layout": "per case the layout kmq_preferred_layout names (see per_case), packed once by "
+                                    "kmq_pack before the timed region"},
         "frac_of_measured_hbm": round(value / world / peak_gbs, 4),
         "us_per_call_mean": round(elapsed_ms * 1e3 / args.steps / step_calls, 3),
         "per_case": per_case,
@@ -515,6 +535,9 @@ def main():
     ap.add_argument("--impl", default="kmq", choices=["kmq", "reference"])
     ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS))
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--case", default="", help='subset of the workload, e.g. "bits=1,M=1" (keys: layer, N, K, bits, M)')
+    ap.add_argument("--layout", default="auto", choices=["auto", "tuned", "table", "canonical"],
+                    help="packed layout of the weights (auto = kmq_preferred_layout per case)")
     ap.add_argument("--quick", action="store_true",
                     help="kernel timing only (no end-to-end leg, CPU baseline or parity check): for profiler runs")
     args = ap.parse_args()

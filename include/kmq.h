@@ -41,8 +41,20 @@
  *       bits = 4: field i at bits [4i, 4i+4) (as canonical);
  *       bits = 2: field i = 4p + c (p, c in 0..3) at bits [2p + 8c, 2p + 8c + 2);
  *       bits = 1: field i = 2c at bit 15 - c, field i = 2c + 1 at bit 31 - c.
- *     Every entry point accepts either layout; kmq_pack writes the one asked
- *     for, the others must be told which one `packed` is in.
+ *     KMQ_LAYOUT_TABLE (what the activation-table kernel reads: b = 1, 2 at
+ *     the smallest batches; for bits = 4 it is identical to KMQ_LAYOUT_TUNED):
+ *     bit planes.  Plane p holds bit p of every index, one byte per group of 8
+ *     consecutive weights of a row, weight 8g + t in bit t.  Rows are grouped
+ *     in tiles of 16 and the groups of a row in chunks of 32 (256 weights);
+ *     with chunks = ceil(K/256), plane p of chunk c of tile T is one
+ *     contiguous 512-byte unit at byte ((T*chunks + c)*bits + p)*512, and
+ *     inside a unit the byte of row n, group g is at
+ *       (2*(n%16) + g%2)*16 + ((g%32)/2 - n%16) mod 16.
+ *     Rows beyond N and groups beyond K are zero padding.
+ *     kmq_packed_bit_index() gives the position of any index bit in any layout.
+ *     Every entry point accepts every layout; kmq_pack writes the one asked
+ *     for, the others must be told which one `packed` is in.  Which layout is
+ *     fastest depends on the batch: kmq_preferred_layout().
  *   - All device pointers must be 16-byte aligned.
  */
 #ifndef KMQ_H_
@@ -69,7 +81,8 @@ typedef enum {
 
 typedef enum {
   KMQ_LAYOUT_CANONICAL = 0,
-  KMQ_LAYOUT_TUNED = 1
+  KMQ_LAYOUT_TUNED = 1,
+  KMQ_LAYOUT_TABLE = 2
 } kmq_layout;
 
 /* Library version (major*10000 + minor*100 + patch). */
@@ -88,6 +101,17 @@ size_t kmq_packed_bytes(int64_t N, int64_t K, int bits, int layout);
  * (index idx[n, j*(32/bits) + i]) inside that word.  -1 for invalid arguments. */
 int64_t kmq_packed_word_index(int64_t n, int64_t j, int64_t N, int64_t K, int bits, int layout);
 int kmq_packed_field_shift(int i, int bits, int layout);
+
+/* Position, in bits from the start of the packed buffer (bit b of byte B is
+ * position 8B + b; bytes of a 32-bit word little-endian), of bit `plane`
+ * (0 = least significant) of idx[n, k].  Valid for every layout; the two
+ * functions above describe the word-based layouts only and return -1 for
+ * KMQ_LAYOUT_TABLE at bits = 1, 2.  -1 for invalid arguments. */
+int64_t kmq_packed_bit_index(int64_t n, int64_t k, int plane, int64_t N, int64_t K, int bits, int layout);
+
+/* The layout in which kmq_linear is fastest for this shape and batch on the
+ * current device (KMQ_LAYOUT_TABLE or KMQ_LAYOUT_TUNED). */
+int kmq_preferred_layout(int64_t N, int64_t K, int bits, int64_t M);
 
 /* Bytes of scratch kmq_linear needs for this shape on the current device
  * (fp32 partial sums of a split along K); may be 0. */
@@ -126,7 +150,14 @@ kmq_status kmq_unpack(const uint32_t* packed, int64_t N, int64_t K, int bits, in
  *   y         DEVICE bf16 [M, N] row-major, fully overwritten.
  *   workspace DEVICE, at least kmq_workspace_bytes(N,K,bits,M,layout) bytes; may be
  *             NULL when that is 0.  Contents on entry are ignored, contents on
- *             return are unspecified.
+ *             return are unspecified.  Calls that share a workspace must not
+ *             overlap on the GPU.
+ *   packed and codebooks are treated as constants of the layer: the kernels
+ *             may read them before earlier work on `stream` has finished
+ *             (programmatic dependent launch).  Earlier kernels of this
+ *             library and ordinary kernels that write them are still ordered
+ *             before the read; a foreign kernel that itself signals an early
+ *             launch of its dependents must not be the one that writes them.
  * The order of the fp32 summation is fixed for a given shape and device, so
  * repeated calls give bit-identical results.  Outputs for non-finite inputs
  * are unspecified.
@@ -208,6 +239,7 @@ kmq_status kmq_linear_tcgen05(const uint32_t* packed, const uint16_t* codebooks,
  * Errors: KMQ_ERR_NULL, KMQ_ERR_CUDA.
  */
 #define KMQ_DEVICE_ERROR_WAIT_TIMEOUT 1u
+#define KMQ_DEVICE_ERROR_SMEM_WINDOW 2u /* the table kernel found its shared memory outside the fixed address window it needs; it stored nothing */
 kmq_status kmq_device_error_flags(unsigned int* flags);
 
 /*

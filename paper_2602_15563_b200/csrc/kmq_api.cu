@@ -3,6 +3,7 @@
 
 #include "kmq_common.cuh"
 #include "kmq_linear_variants.cuh"
+#include "kmq_table_layout.cuh"
 
 namespace kmq {
 
@@ -28,7 +29,11 @@ const DeviceInfo* device_info() {
 namespace {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-inline bool known_layout(int layout) { return layout == KMQ_LAYOUT_CANONICAL || layout == KMQ_LAYOUT_TUNED; }
+inline bool known_layout(int layout) {
+  return layout == KMQ_LAYOUT_CANONICAL || layout == KMQ_LAYOUT_TUNED || layout == KMQ_LAYOUT_TABLE;
+}
+// b = 4 is stored identically in the tuned and the table layout
+inline bool is_plane_layout(int layout, int bits) { return layout == KMQ_LAYOUT_TABLE && bits != 4; }
 
 kmq_status check_shape(int64_t N, int64_t K, int bits, int64_t M) {
   if (bits != 1 && bits != 2 && bits != 4) return KMQ_ERR_BITS;
@@ -66,21 +71,33 @@ const char* kmq_status_string(int status) {
 size_t kmq_packed_bytes(int64_t N, int64_t K, int bits, int layout) {
   if (!known_layout(layout) || check_shape(N, K, bits, 1) != KMQ_OK) return 0;
   const int64_t wpr = K / (32 / bits);
-  if (layout == KMQ_LAYOUT_TUNED) return (size_t)tuned_total_words(N, wpr) * 4u;
+  if (is_plane_layout(layout, bits)) return (size_t)table_total_bytes(N, K, bits);
+  if (layout != KMQ_LAYOUT_CANONICAL) return (size_t)tuned_total_words(N, wpr) * 4u;
   return (size_t)N * (size_t)wpr * 4u;
 }
 
 int64_t kmq_packed_word_index(int64_t n, int64_t j, int64_t N, int64_t K, int bits, int layout) {
   if (!known_layout(layout) || check_shape(N, K, bits, 1) != KMQ_OK) return -1;
   const int64_t wpr = K / (32 / bits);
-  if (n < 0 || n >= N || j < 0 || j >= wpr) return -1;
-  return layout == KMQ_LAYOUT_TUNED ? tuned_word_index(n, j, tuned_steps(wpr)) : n * wpr + j;
+  if (n < 0 || n >= N || j < 0 || j >= wpr || is_plane_layout(layout, bits)) return -1;
+  return layout != KMQ_LAYOUT_CANONICAL ? tuned_word_index(n, j, tuned_steps(wpr)) : n * wpr + j;
 }
 
 int kmq_packed_field_shift(int i, int bits, int layout) {
   if (!known_layout(layout) || (bits != 1 && bits != 2 && bits != 4) || i < 0 || i >= 32 / bits) return -1;
-  const bool tuned = layout == KMQ_LAYOUT_TUNED;
+  if (is_plane_layout(layout, bits)) return -1;
+  const bool tuned = layout != KMQ_LAYOUT_CANONICAL;
   return bits == 1 ? field_pos<1>(i, tuned) : bits == 2 ? field_pos<2>(i, tuned) : field_pos<4>(i, tuned);
+}
+
+int64_t kmq_packed_bit_index(int64_t n, int64_t k, int plane, int64_t N, int64_t K, int bits, int layout) {
+  if (!known_layout(layout) || check_shape(N, K, bits, 1) != KMQ_OK) return -1;
+  if (n < 0 || n >= N || k < 0 || k >= K || plane < 0 || plane >= bits) return -1;
+  if (is_plane_layout(layout, bits))
+    return table_byte_offset(n, k >> 3, plane, table_chunks(K), bits) * 8 + (k & 7);
+  const int64_t per = 32 / bits, wpr = K / per;
+  const int64_t word = layout != KMQ_LAYOUT_CANONICAL ? tuned_word_index(n, k / per, tuned_steps(wpr)) : n * wpr + k / per;
+  return word * 32 + kmq_packed_field_shift((int)(k % per), bits, layout) + plane;
 }
 
 size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M, int layout) {
@@ -91,6 +108,11 @@ size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M, int layout
 int kmq_linear_num_launches(int64_t N, int64_t K, int bits, int64_t M, int layout) {
   if (!known_layout(layout) || check_shape(N, K, bits, M) != KMQ_OK) return 0;
   return plan_linear(N, K, bits, M, layout).launches;
+}
+
+int kmq_preferred_layout(int64_t N, int64_t K, int bits, int64_t M) {
+  if (check_shape(N, K, bits, M) != KMQ_OK) return KMQ_LAYOUT_TUNED;
+  return linear_lut_preferred(N, K, bits, M) ? KMQ_LAYOUT_TABLE : KMQ_LAYOUT_TUNED;
 }
 
 const char* kmq_linear_variant(int64_t N, int64_t K, int bits, int64_t M, int layout) {

@@ -3,6 +3,7 @@
 // produces exactly one 16-byte store (8 weights) from 8*BITS packed bits and
 // consecutive threads write consecutive 16-byte pieces.
 #include "kmq_common.cuh"
+#include "kmq_table_layout.cuh"
 
 namespace kmq {
 namespace {
@@ -97,16 +98,50 @@ __global__ void __launch_bounds__(256) dequant_rows_kernel(const uint32_t* __res
   }
 }
 
+// Table (bit-plane) layout: a thread gathers the plane bytes of one group of 8 weights, interleaves them into
+// LSB-first index fields and stores the 8 decoded weights as one 16-byte piece.
+template <int BITS>
+__global__ void __launch_bounds__(256) dequant_table_kernel(const uint32_t* __restrict__ packed,
+                                                            const uint16_t* __restrict__ cb, uint16_t* __restrict__ W,
+                                                            int64_t N, int64_t K) {
+  constexpr int Q = 1 << BITS;
+  const uint8_t* bytes = reinterpret_cast<const uint8_t*>(packed);
+  const int gpr = (int)(K >> 3);
+  const int64_t chunks = table_chunks(K);
+  for (int64_t n = blockIdx.x; n < N; n += gridDim.x) {
+    const uint16_t* row_cb = cb + n * Q;
+    uint32_t c0, c1;
+    load_codebook<BITS>(row_cb, c0, c1);
+    uint4* out = reinterpret_cast<uint4*>(W + n * K);
+    for (int g = threadIdx.x; g < gpr; g += 256) {
+      uint32_t v = __ldg(bytes + table_byte_offset(n, g, 0, chunks, BITS));
+      if constexpr (BITS == 2) {
+        const uint32_t hi = __ldg(bytes + table_byte_offset(n, g, 1, chunks, BITS));
+        uint32_t z = 0;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) z |= (((v >> t) & 1u) | (((hi >> t) & 1u) << 1)) << (2 * t);
+        v = z;
+      }
+      stg_stream_u4(out + g, decode8<BITS>(v, c0, c1, row_cb));
+    }
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_dequant(const uint32_t* packed, const uint16_t* cb, uint16_t* W, int64_t N, int64_t K, int bits,
                            int layout, cudaStream_t s) {
   const DeviceInfo* di = device_info();
-  if (!di) return cudaGetLastError();
-  const bool tuned = layout == KMQ_LAYOUT_TUNED;
+  if (!di) return cudaErrorInvalidDevice;
+  const bool tuned = layout != KMQ_LAYOUT_CANONICAL;
   int64_t blocks = N;
   const int64_t cap = (int64_t)di->sm_count * 8;   // 8 resident CTAs of 256 threads per SM
   if (blocks > cap) blocks = cap;
+  if (layout == KMQ_LAYOUT_TABLE && bits != 4) {
+    if (bits == 1) dequant_table_kernel<1><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+    else dequant_table_kernel<2><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
+    return cudaGetLastError();
+  }
   if (bits == 1 && tuned) dequant_rows_kernel<1, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
   else if (bits == 1) dequant_rows_kernel<1, false><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);
   else if (bits == 2 && tuned) dequant_rows_kernel<2, true><<<(int)blocks, 256, 0, s>>>(packed, cb, W, N, K);

@@ -8,6 +8,20 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
   LinearPlan p;
   p.workspace = 0;
   p.split_k = 1;
+  if (layout == KMQ_LAYOUT_TABLE && bits != 4) {
+    if (!linear_lut_supports(N, K, bits, M)) {
+      p.variant = kVariantUnsupported;
+      p.launches = 0;
+      p.name = "unsupported";
+      return p;
+    }
+    p.variant = kVariantLut;
+    p.workspace = linear_lut_scratch_bytes(N, K, bits);
+    p.launches = (int)(p.workspace ? 2 * M : M);
+    p.name = bits == 1 ? "table_lookup_b1" : "table_lookup_b2";
+    return p;
+  }
+  if (layout == KMQ_LAYOUT_TABLE) layout = KMQ_LAYOUT_TUNED;   // b = 4: the two layouts are the same
   if (linear_mma_supports(N, K, bits, M)) {
     const bool tuned = layout == KMQ_LAYOUT_TUNED;
     p.variant = tuned ? kVariantTiled : kVariantMma;
@@ -51,7 +65,12 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
 cudaError_t launch_linear(const LinearPlan& plan, const uint32_t* packed, const uint16_t* cb, const uint16_t* x,
                           uint16_t* y, int64_t N, int64_t K, int bits, int64_t M, int layout, void* workspace,
                           cudaStream_t s) {
+  if (layout == KMQ_LAYOUT_TABLE && bits == 4) layout = KMQ_LAYOUT_TUNED;
   switch (plan.variant) {
+    case kVariantLut:
+      return launch_linear_lut(packed, cb, x, y, N, K, bits, M, workspace, s);
+    case kVariantUnsupported:
+      return cudaErrorNotSupported;
     case kVariantSplit:
       return launch_linear_split(packed, cb, x, y, N, K, bits, M, workspace, plan.split_k, s);
     case kVariantUmma:

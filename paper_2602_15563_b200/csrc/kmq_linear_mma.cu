@@ -14,9 +14,9 @@
 //   b = 4  a per-row table of all 256 (centroid, centroid) pairs in shared
 //          memory, one copy per lane bank so lookups never conflict; one
 //          32-bit LDS yields two weights.
-//   b = 1  W^ = c0 + bit*(c1 - c0): the tensor core multiplies by the signs
-//          (+1 for bit 0, -1 for bit 1) and the codebook is applied once per
-//          output in the epilogue from D = sum(+-x) and S = sum(x).
+//   b = 1  a shift puts two index bits on bits 15 and 31, a sign-replicating
+//          PRMT spreads them over their half words and one LOP3 selects c0 or
+//          c1: bit copies of the stored centroids.
 // The order in which a word's fields reach the k-slots of an MMA is whatever
 // is cheapest to extract; the activations are staged in shared memory in that
 // same order, so the canonical packed layout is consumed as is.
@@ -46,7 +46,7 @@ struct Geo {
 
 template <int BITS, int MMAX>
 constexpr int smem_bytes() {
-  return Geo<BITS>::kTableBytes + kWarps * MMAX * Geo<BITS>::kRowStride + kRedBytes + 16 * kWarps * 4;
+  return Geo<BITS>::kTableBytes + kWarps * MMAX * Geo<BITS>::kRowStride + kRedBytes;
 }
 
 // ---------------------------------------------------------------------------
@@ -120,11 +120,10 @@ __global__ void __launch_bounds__(kThreads) linear_mma_kernel(const uint32_t* __
   using G = Geo<BITS>;
   constexpr int Q = G::kMmaPerWord;
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  // [pair tables (b = 4)] [staged activations: kWarps x MMAX rows] [warp partials] [S partials (b = 1)]
+  // [pair tables (b = 4)] [staged activations: kWarps x MMAX rows] [warp partials]
   unsigned char* const tables = smem_raw;
   unsigned char* const xs_all = smem_raw + G::kTableBytes;
   float* const red = reinterpret_cast<float*>(xs_all + kWarps * MMAX * G::kRowStride);
-  float* const red_s = red + kWarps * 32 * 4;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -150,6 +149,11 @@ __global__ void __launch_bounds__(kThreads) linear_mma_kernel(const uint32_t* __
   }
 
   // ---- per-row decode state ----
+  Dec1 sg, sh;
+  if constexpr (BITS == 1) {
+    sg.init(cb + rg * 2);
+    sh.init(cb + rh * 2);
+  }
   Dec2 dg, dh;
   if constexpr (BITS == 2) {
     dg.init(cb + rg * 4);
@@ -170,9 +174,6 @@ __global__ void __launch_bounds__(kThreads) linear_mma_kernel(const uint32_t* __
   const uint32_t lane4 = lane * 4;
 
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  float sacc[MMAX];   // b = 1 only: partial sums of the activations of batch row m
-#pragma unroll
-  for (int m = 0; m < MMAX; ++m) sacc[m] = 0.f;
 
   const unsigned char* const xb_lane = xs_warp + g * G::kRowStride + t * 8;   // B fragments: batch row g, chunk t
   const bool has_col = g < M;
@@ -216,47 +217,21 @@ __global__ void __launch_bounds__(kThreads) linear_mma_kernel(const uint32_t* __
               a1 = *reinterpret_cast<const uint32_t*>(tables + kPairTableBytes + ob0);
               a3 = *reinterpret_cast<const uint32_t*>(tables + kPairTableBytes + ob1);
             } else {
-              // pair c = 2q: weights (15-2q | 31-2q); pair c = 2q+1: weights (14-2q | 30-2q); sign set <=> bit set
-              a0 = ((wa[j] << (2 * q)) & 0x80008000u) | 0x3F803F80u;
-              a2 = ((wa[j] << (2 * q + 1)) & 0x80008000u) | 0x3F803F80u;
-              a1 = ((wb[j] << (2 * q)) & 0x80008000u) | 0x3F803F80u;
-              a3 = ((wb[j] << (2 * q + 1)) & 0x80008000u) | 0x3F803F80u;
+              // pair c = 2q: weights (15-2q | 31-2q); pair c = 2q+1: weights (14-2q | 30-2q) on bits 15 and 31
+              a0 = sg.select(wa[j] << (2 * q));
+              a2 = sg.select(wa[j] << (2 * q + 1));
+              a1 = sh.select(wb[j] << (2 * q));
+              a3 = sh.select(wb[j] << (2 * q + 1));
             }
             mma_bf16_16816(acc, a0, a1, a2, a3, b.x, b.y);
-          }
-        }
-        if constexpr (BITS == 1) {
-          // S[m] = sum_k x[m,k].  The 512 staged activations of a batch row, read as two 16x16 A tiles and
-          // multiplied by a matrix of ones, give 16 row sums per tile; their total is order-independent.
-#pragma unroll
-          for (int m = 0; m < MMAX; ++m) {
-            if (m < M) {
-#pragma unroll
-              for (int h = 0; h < 2; ++h) {
-                const uint4 v = *reinterpret_cast<const uint4*>(xs_warp + m * G::kRowStride + h * 512 + lane * 16);
-                float tmp[4] = {0.f, 0.f, 0.f, 0.f};
-                mma_bf16_16816(tmp, v.x, v.y, v.z, v.w, 0x3F803F80u, 0x3F803F80u);
-                sacc[m] += tmp[0] + tmp[2];   // rows g and g + 8 (identical in every column)
-              }
-            }
           }
         }
       }
     }
   }
 
-  // ---- add the partial sums of the warps, apply the codebook (b = 1), store ----
+  // ---- add the partial sums of the warps, store ----
   *reinterpret_cast<float4*>(red + (warp * 32 + lane) * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-  if constexpr (BITS == 1) {
-#pragma unroll
-    for (int m = 0; m < MMAX; ++m) {
-      float v = sacc[m];
-      v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
-      v += __shfl_xor_sync(0xFFFFFFFFu, v, 8);
-      v += __shfl_xor_sync(0xFFFFFFFFu, v, 16);
-      if (lane == 0) red_s[warp * MMAX + m] = v;   // lanes with t = 0 cover every row once
-    }
-  }
   __syncthreads();
   if (threadIdx.x < kRows * 8) {
     const int r = threadIdx.x & 15, m = threadIdx.x >> 4;   // consecutive threads -> consecutive output rows
@@ -266,16 +241,6 @@ __global__ void __launch_bounds__(kThreads) linear_mma_kernel(const uint32_t* __
       float v = 0.f;
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) v += red[(w * 32 + src_lane) * 4 + src_reg];
-      if constexpr (BITS == 1) {
-        float s = 0.f;
-        const int mm = m < MMAX ? m : 0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) s += red_s[w * MMAX + mm];
-        // v = T0 - T1, s = T0 + T1 with T_i the sum of the activations whose weight has index i
-        const uint32_t c = __ldg(reinterpret_cast<const uint32_t*>(cb + n * 2));
-        const float c0 = bf16_bits_to_float(c & 0xFFFFu), c1 = bf16_bits_to_float(c >> 16);
-        v = fmaf(c0, 0.5f * (s + v), c1 * (0.5f * (s - v)));
-      }
       y[(int64_t)m * N + n] = (uint16_t)float_to_bf16_bits(v);
     }
   }

@@ -43,8 +43,7 @@ struct MSmem {
   static constexpr int kBuf = 8 * NT * G::kRowStride;                 // one x buffer: 8 NT batch rows of one step
   static constexpr int kX = kGroups * 2 * kBuf;                       // double buffered, per K-group
   static constexpr int kRed = (kGroups - 1) * TPC * 32 * NT * 4 * 4;  // accumulators of K-groups 1.. (aliases x)
-  static constexpr int kSums = kGroups * 8 * NT * 4;                  // b = 1: sum of x per batch row and K-group
-  static constexpr int kTotal = kTableBytes + (kX > kRed ? kX : kRed) + kSums;
+  static constexpr int kTotal = kTableBytes + (kX > kRed ? kX : kRed);
 };
 
 template <int BITS>
@@ -76,12 +75,10 @@ __global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 
   constexpr int kThreads = W * 32;
   constexpr int Q = G::kMmaPerWord;
   constexpr int kGroups = SM::kGroups, kGroupThreads = TPC * 32;
-  constexpr int kSumRows = 8 * NT / TPC;   // b = 1: batch rows whose activations one warp sums
   extern __shared__ __align__(128) unsigned char smem_raw[];
   unsigned char* const tables = smem_raw;
   unsigned char* const xbase = smem_raw + SM::kTableBytes;
   float* const red = reinterpret_cast<float*>(xbase);                       // reused after the main loop
-  float* const sums = reinterpret_cast<float*>(xbase + (SM::kX > SM::kRed ? SM::kX : SM::kRed));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -125,6 +122,11 @@ __global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 
   if (group < steps) stage(group, 0);
 
   // ---- per-row decode state ----
+  Dec1 sg, sh;
+  if constexpr (BITS == 1) {
+    sg.init(cb + min(row0 + g, N - 1) * 2);
+    sh.init(cb + min(row0 + g + 8, N - 1) * 2);
+  }
   Dec2 dg, dh;
   if constexpr (BITS == 2) {
     dg.init(cb + min(row0 + g, N - 1) * 4);
@@ -146,10 +148,6 @@ __global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 
   float acc[NT][4];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-  // b = 1: warp wt of a K-group sums the activations of batch rows m = wt, wt + TPC, ...
-  float sacc[kSumRows];
-#pragma unroll
-  for (int i = 0; i < kSumRows; ++i) sacc[i] = 0.f;
 
   for (int s0 = group; s0 < steps; s0 += 2 * kGroups) {   // uniform over the K-group
 #pragma unroll
@@ -201,10 +199,10 @@ __global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 
               a3 = prmt(hi[2], hi[3], 0x7610u);
             } else {
               const uint32_t m0 = kPow2[2 * q], m1 = kPow2[2 * q + 1];
-              a0 = and_or(wa[j] * m0, 0x80008000u, 0x3F803F80u);
-              a2 = and_or(wa[j] * m1, 0x80008000u, 0x3F803F80u);
-              a1 = and_or(wb[j] * m0, 0x80008000u, 0x3F803F80u);
-              a3 = and_or(wb[j] * m1, 0x80008000u, 0x3F803F80u);
+              a0 = sg.select(wa[j] * m0);
+              a2 = sg.select(wa[j] * m1);
+              a1 = sh.select(wb[j] * m0);
+              a3 = sh.select(wb[j] * m1);
             }
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
@@ -213,36 +211,10 @@ __global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 
         }
       }
     }
-    if constexpr (BITS == 1) {
-      // S[m] = sum_k x[m,k]: the 512 staged activations of a batch row as two 16x16 A tiles times ones
-#pragma unroll
-      for (int i = 0; i < kSumRows; ++i) {
-        const int m = wt + TPC * i;
-        if (m < M) {
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const uint4 v = *reinterpret_cast<const uint4*>(xs + m * G::kRowStride + piece_offset<BITS>(lane + 32 * h));
-            float tmp[4] = {0.f, 0.f, 0.f, 0.f};
-            mma_bf16_16816(tmp, v.x, v.y, v.z, v.w, 0x3F803F80u, 0x3F803F80u);
-            sacc[i] += tmp[0] + tmp[2];
-          }
-        }
-      }
-    }
    }
   }
 
-  // ---- K-groups 1.. hand their partial sums to K-group 0, which adds, applies the codebook (b = 1) and stores ----
-  if constexpr (BITS == 1) {
-#pragma unroll
-    for (int i = 0; i < kSumRows; ++i) {
-      float v = sacc[i];
-      v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
-      v += __shfl_xor_sync(0xFFFFFFFFu, v, 8);
-      v += __shfl_xor_sync(0xFFFFFFFFu, v, 16);
-      if (lane == 0) sums[group * 8 * NT + wt + TPC * i] = v;   // lanes with t = 0 cover every row once
-    }
-  }
+  // ---- K-groups 1.. hand their partial sums to K-group 0, which adds and stores ----
   __syncthreads();   // every warp is done with the x buffers; `red` aliases them
   if (group > 0) {
 #pragma unroll
@@ -252,11 +224,6 @@ __global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 
   }
   __syncthreads();
   if (group == 0 && has_tile) {
-    uint32_t cw0 = 0, cw1 = 0;
-    if constexpr (BITS == 1) {
-      cw0 = __ldg(reinterpret_cast<const uint32_t*>(cb + min(row0 + g, N - 1) * 2));
-      cw1 = __ldg(reinterpret_cast<const uint32_t*>(cb + min(row0 + g + 8, N - 1) * 2));
-    }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       float v[4] = {acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]};
@@ -270,18 +237,7 @@ __global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 
       for (int r = 0; r < 4; ++r) {
         const int m = nt * 8 + 2 * t + (r & 1);
         const int64_t n = row0 + g + 8 * (r >> 1);
-        if (m < M && n < N) {
-          float out = v[r];
-          if constexpr (BITS == 1) {
-            float sx = 0.f;
-#pragma unroll
-            for (int gq = 0; gq < kGroups; ++gq) sx += sums[gq * 8 * NT + m];
-            const uint32_t c = (r >> 1) ? cw1 : cw0;
-            const float c0 = bf16_bits_to_float(c & 0xFFFFu), c1 = bf16_bits_to_float(c >> 16);
-            out = fmaf(c0, 0.5f * (sx + out), c1 * (0.5f * (sx - out)));
-          }
-          y[(int64_t)m * N + n] = (uint16_t)float_to_bf16_bits(out);
-        }
+        if (m < M && n < N) y[(int64_t)m * N + n] = (uint16_t)float_to_bf16_bits(v[r]);
       }
     }
   }

@@ -13,9 +13,8 @@
 //   b = 4  per-row table of all 256 (centroid, centroid) pairs in shared memory, one copy per lane bank; the
 //          byte offset of a lookup is one PRMT of the packed word, one 32-bit LDS yields two weights.
 //   b = 2  the row's 4 centroids are the 8 source bytes of one PRMT; one PRMT yields two weights.
-//   b = 1  W^ = c0 + bit * (c1 - c0): the MMA multiplies by the signs (+1 / -1, one LOP3 per two weights, the
-//          shifts as multiplies on the FMA pipe) and the codebook is applied per output in the epilogue from
-//          D = sum(+-x) and S = sum(x).
+//   b = 1  a shift (as a multiply on the FMA pipe) puts two index bits on bits 15 and 31, a sign-replicating PRMT
+//          spreads them over their half words and one LOP3 selects c0 or c1: bit copies of the stored centroids.
 #include "kmq_common.cuh"
 #include "kmq_linear_variants.cuh"
 #include "kmq_mma_common.cuh"
@@ -59,8 +58,7 @@ struct TSmem {
   using G = TGeo<BITS>;
   static constexpr int kXs = kWarps * MMAX * G::kRowStride;
   static constexpr int kRed = kWarps * 32 * 16;
-  static constexpr int kRedS = kWarps * MMAX * 4;
-  static constexpr int kTotal = G::kTableBytes + kXs + kRed + kRedS;
+  static constexpr int kTotal = G::kTableBytes + kXs + kRed;
 };
 
 // shared-memory byte offset (within one batch row of a warp's slice) of 16-byte piece `w` of a step
@@ -72,12 +70,12 @@ __device__ __forceinline__ int piece_offset(int w) {
 }
 
 // Steps [sa, sb) of tile `tile_id`, all 8 warps of the CTA: on return thread i < 128 holds in `v` the sum over those
-// steps for output row i % 16 and batch row i / 16 (b = 1: the signed sum D, and in `sx` the sum of the activations
-// under those steps).  May be called several times by one CTA; shared memory is reused from call to call.
+// steps for output row i % 16 and batch row i / 16.  May be called several times by one CTA; shared memory is reused
+// from call to call.
 template <int BITS, int MMAX>
 __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed, const uint16_t* __restrict__ cb,
                                              const uint16_t* __restrict__ x, int64_t N, int64_t K, int M,
-                                             int64_t tile_id, int sa, int sb, float& v, float& sx) {
+                                             int64_t tile_id, int sa, int sb, float& v) {
   using G = TGeo<BITS>;
   using SM = TSmem<BITS, MMAX>;
   constexpr int Q = G::kMmaPerWord;
@@ -91,7 +89,6 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
   unsigned char* const tables = smem_raw;
   unsigned char* const xs_warp = smem_raw + G::kTableBytes + (threadIdx.x >> 5) * (MMAX * G::kRowStride);
   float* const red = reinterpret_cast<float*>(smem_raw + G::kTableBytes + SM::kXs);
-  float* const red_s = red + kWarps * 32 * 4;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -139,6 +136,11 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
   }
 
   // ---- per-row decode state ----
+  Dec1 sg, sh;
+  if constexpr (BITS == 1) {
+    sg.init(cb + min(row0 + g, N - 1) * 2);
+    sh.init(cb + min(row0 + g + 8, N - 1) * 2);
+  }
   Dec2 dg, dh;
   if constexpr (BITS == 2) {
     dg.init(cb + min(row0 + g, N - 1) * 4);
@@ -167,9 +169,6 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
   const uint32_t lane4 = lane * 4;
 
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  float sacc[MMAX];
-#pragma unroll
-  for (int m = 0; m < MMAX; ++m) sacc[m] = 0.f;
 
   // B fragments: lane (g, t) supplies batch row g; the columns of an MMA are independent, so lanes with
   // g >= M re-read the last real row and their columns are never stored.
@@ -216,29 +215,12 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
               } else {
                 // shift by c puts weights (2c, 2c+1) of the word on the two sign bits; c = 2q and 2q + 1
                 const uint32_t m0 = kPow2[2 * q], m1 = kPow2[2 * q + 1];
-                a0 = and_or(wa[j] * m0, 0x80008000u, 0x3F803F80u);
-                a2 = and_or(wa[j] * m1, 0x80008000u, 0x3F803F80u);
-                a1 = and_or(wb[j] * m0, 0x80008000u, 0x3F803F80u);
-                a3 = and_or(wb[j] * m1, 0x80008000u, 0x3F803F80u);
+                a0 = sg.select(wa[j] * m0);
+                a2 = sg.select(wa[j] * m1);
+                a1 = sh.select(wb[j] * m0);
+                a3 = sh.select(wb[j] * m1);
               }
               mma_bf16_16816(acc, a0, a1, a2, a3, qq ? xv.z : xv.x, qq ? xv.w : xv.y);
-            }
-          }
-        }
-        if constexpr (BITS == 1) {
-          // S[m] = sum_k x[m,k]: the 512 staged activations of a batch row as two 16x16 A tiles times a matrix
-          // of ones give 16 row sums each; the order of the addends is irrelevant.
-#pragma unroll
-          for (int m = 0; m < MMAX; ++m) {
-            if (m < M) {
-#pragma unroll
-              for (int h = 0; h < 2; ++h) {
-                const uint4 v =
-                    *reinterpret_cast<const uint4*>(xs_warp + m * G::kRowStride + piece_offset<BITS>(lane + 32 * h));
-                float tmp[4] = {0.f, 0.f, 0.f, 0.f};
-                mma_bf16_16816(tmp, v.x, v.y, v.z, v.w, 0x3F803F80u, 0x3F803F80u);
-                sacc[m] += tmp[0] + tmp[2];   // rows g and g + 8 (identical in every column)
-              }
             }
           }
         }
@@ -253,61 +235,25 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
     }
   }
 
-  // ---- add the partial sums of the warps, apply the codebook (b = 1), store ----
+  // ---- add the partial sums of the warps ----
   *reinterpret_cast<float4*>(red + (warp * 32 + lane) * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-  if constexpr (BITS == 1) {
-#pragma unroll
-    for (int m = 0; m < MMAX; ++m) {
-      float v = sacc[m];
-      v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
-      v += __shfl_xor_sync(0xFFFFFFFFu, v, 8);
-      v += __shfl_xor_sync(0xFFFFFFFFu, v, 16);
-      if (lane == 0) red_s[warp * MMAX + m] = v;   // lanes with t = 0 cover every row once
-    }
-  }
   __syncthreads();
   v = 0.f;
-  sx = 0.f;
   if (threadIdx.x < kRows * 8) {
     const int r = threadIdx.x & 15, m = threadIdx.x >> 4;   // consecutive threads -> consecutive output rows
     const int src_lane = (r & 7) * 4 + (m >> 1), src_reg = (r >> 3) * 2 + (m & 1);
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) v += red[(w * 32 + src_lane) * 4 + src_reg];
-    if constexpr (BITS == 1) {
-      const int mm = m < MMAX ? m : 0;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) sx += red_s[w * MMAX + mm];
-    }
   }
 }
 
-// Thread i < 128: apply the codebook (b = 1) to the finished sum of output row row0 + i % 16, batch row i / 16, and
-// store it as bf16.  `cb1` = the two centroids of that row (b = 1 only).
-template <int BITS>
-__device__ __forceinline__ void store_output(float v, float sx, uint32_t cb1, uint16_t* __restrict__ y, int64_t N,
-                                             int M, int64_t row0) {
+// Thread i < 128: store the finished sum of output row row0 + i % 16, batch row i / 16, as bf16.
+__device__ __forceinline__ void store_output(float v, uint16_t* __restrict__ y, int64_t N, int M, int64_t row0) {
   if (threadIdx.x < kRows * 8) {
     const int r = threadIdx.x & 15, m = threadIdx.x >> 4;
     const int64_t n = row0 + r;
-    if (m < M && n < N) {
-      if constexpr (BITS == 1) {
-        // v = T0 - T1, sx = T0 + T1 with T_i the sum of the activations whose weight has index i
-        const float c0 = bf16_bits_to_float(cb1 & 0xFFFFu), c1 = bf16_bits_to_float(cb1 >> 16);
-        v = fmaf(c0, 0.5f * (sx + v), c1 * (0.5f * (sx - v)));
-      }
-      y[(int64_t)m * N + n] = (uint16_t)float_to_bf16_bits(v);
-    }
+    if (m < M && n < N) y[(int64_t)m * N + n] = (uint16_t)float_to_bf16_bits(v);
   }
-}
-
-// b = 1: the two centroids of the output row thread i < 128 will store; fetched early, off the critical path.
-template <int BITS>
-__device__ __forceinline__ uint32_t load_cb1(const uint16_t* __restrict__ cb, int64_t N, int64_t row0) {
-  if constexpr (BITS == 1) {
-    if (threadIdx.x < kRows * 8)
-      return __ldg(reinterpret_cast<const uint32_t*>(cb + min(row0 + (threadIdx.x & 15), N - 1) * 2));
-  }
-  return 0;
 }
 
 // One CTA per tile.
@@ -325,13 +271,12 @@ __global__ void __launch_bounds__(kThreads, KMQ_TILED_MINB) linear_tiled_kernel(
 #endif
   const int steps = (int)((K / (4 * TGeo<BITS>::kWordK) + 3) >> 2);
   const int64_t row0 = (int64_t)blockIdx.x * kRows;
-  const uint32_t cb1 = load_cb1<BITS>(cb, N, row0);
-  float v, sx;
-  tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, blockIdx.x, 0, steps, v, sx);
+  float v;
+  tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, blockIdx.x, 0, steps, v);
 #if KMQ_PDL
   asm volatile("griddepcontrol.launch_dependents;");
 #endif
-  store_output<BITS>(v, sx, cb1, y, N, M, row0);
+  store_output(v, y, N, M, row0);
 }
 
 // ---------------------------------------------------------------------------
@@ -341,7 +286,7 @@ __global__ void __launch_bounds__(kThreads, KMQ_TILED_MINB) linear_tiled_kernel(
 // tiles, one at each end; their sums go to scratch slot [cta][0] (range starts inside the tile) or [cta][1] (range
 // ends inside it).  Every cut therefore has exactly two contributors, which the fix-up kernel adds in a fixed order.
 // ---------------------------------------------------------------------------
-constexpr int kSlotFloats = kRows * 8 + 8;   // 128 sums + 8 sums of x (b = 1)
+constexpr int kSlotFloats = kRows * 8 + 8;   // 128 sums (+ 8 unused: keeps the slots 32-byte aligned)
 
 template <int BITS, int MMAX>
 __global__ void __launch_bounds__(kThreads, KMQ_TILED_MINB) linear_split_kernel(const uint32_t* __restrict__ packed,
@@ -355,15 +300,13 @@ __global__ void __launch_bounds__(kThreads, KMQ_TILED_MINB) linear_split_kernel(
   for (int64_t tile = u0 / steps; tile * steps < u1; ++tile) {
     const int64_t base = tile * steps;
     const int sa = (int)(u0 > base ? u0 - base : 0), sb = (int)(u1 - base < steps ? u1 - base : steps);
-    const uint32_t cb1 = load_cb1<BITS>(cb, N, tile * kRows);
-    float v, sx;
-    tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, tile, sa, sb, v, sx);
+    float v;
+    tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, tile, sa, sb, v);
     if (sa == 0 && sb == steps) {
-      store_output<BITS>(v, sx, cb1, y, N, M, tile * kRows);
+      store_output(v, y, N, M, tile * kRows);
     } else if (threadIdx.x < kRows * 8) {
       float* slot = scratch + ((int64_t)blockIdx.x * 2 + (sa == 0 ? 1 : 0)) * kSlotFloats;
       slot[threadIdx.x] = v;
-      if (BITS == 1 && (threadIdx.x & 15) == 0) slot[kRows * 8 + (threadIdx.x >> 4)] = sx;
     }
   }
 }
@@ -381,11 +324,8 @@ __global__ void __launch_bounds__(kRows * 8) linear_split_fixup_kernel(const flo
   const int64_t row0 = (cut / steps) * kRows;
   const float* end_of_c = scratch + ((int64_t)blockIdx.x * 2 + 1) * kSlotFloats;
   const float* start_of_next = scratch + ((int64_t)(blockIdx.x + 1) * 2) * kSlotFloats;
-  const int m = threadIdx.x >> 4;
   const float v = end_of_c[threadIdx.x] + start_of_next[threadIdx.x];
-  float sx = 0.f;
-  if constexpr (BITS == 1) sx = end_of_c[kRows * 8 + m] + start_of_next[kRows * 8 + m];
-  store_output<BITS>(v, sx, load_cb1<BITS>(cb, N, row0), y, N, M, row0);
+  store_output(v, y, N, M, row0);
 }
 
 template <int BITS, int MMAX>

@@ -638,8 +638,15 @@ cudaError_t read_device_error_flags(unsigned int* flags) {
   if (e != cudaSuccess) return e;
   e = cudaMemcpyFromSymbol(flags, g_device_error_flags, sizeof(unsigned int));
   if (e != cudaSuccess) return e;
-  const unsigned int zero = 0;
-  return cudaMemcpyToSymbol(g_device_error_flags, &zero, sizeof(unsigned int));
+  if (*flags) {
+    const unsigned int zero = 0;
+    e = cudaMemcpyToSymbol(g_device_error_flags, &zero, sizeof(unsigned int));
+    if (e != cudaSuccess) return e;
+  }
+  unsigned int lut = 0;
+  e = read_lut_error_flags(&lut);
+  *flags |= lut;
+  return e;
 }
 
 

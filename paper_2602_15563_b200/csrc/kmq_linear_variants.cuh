@@ -13,6 +13,8 @@ enum LinearVariant : int {
   kVariantUmma = 5,      // tuned layout, M > 32 and enough 128-row blocks to fill the SMs: tcgen05.mma, weights
                          // dequantised into tensor memory
   kVariantSplit = 4,     // tuned layout, M <= 8, more tiles than resident CTAs: equal step ranges + fix-up (scratch)
+  kVariantLut = 6,       // table layout, b = 1, 2: activation tables in shared memory, one lookup per 8 weights (scratch)
+  kVariantUnsupported = 7,
 };
 
 cudaError_t launch_linear_generic(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
@@ -37,6 +39,12 @@ int linear_umma_rows_per_launch();
 int linear_umma_ksplit(int64_t N, int64_t K, int bits, int batch);   // CTAs (cluster size) per 128-row block
 cudaError_t launch_linear_umma(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                                int64_t K, int bits, int64_t M, cudaStream_t s);
+bool linear_lut_supports(int64_t N, int64_t K, int bits, int64_t M);
+bool linear_lut_preferred(int64_t N, int64_t K, int bits, int64_t M);   // faster than the tensor-core kernels here
+size_t linear_lut_scratch_bytes(int64_t N, int64_t K, int bits);
+cudaError_t launch_linear_lut(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
+                              int64_t K, int bits, int64_t M, void* scratch, cudaStream_t s);
+cudaError_t read_lut_error_flags(unsigned int* flags);   // reads and clears the table kernel's error word
 cudaError_t read_device_error_flags(unsigned int* flags);   // synchronises; reads and clears the sticky error word
 
 }  // namespace kmq

@@ -25,6 +25,24 @@ __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
   return d;
 }
 
+// b = 1: the two centroids of one row as bf16 pairs (c0, c0) and (c0 ^ c1, c0 ^ c1).  select() turns a word whose
+// bits 15 and 31 are two index bits into the two weights, each a bit copy of a stored centroid: a sign-replicating
+// PRMT spreads each bit over its half word, one LOP3 flips c0 into c1 where the bit is set.
+struct Dec1 {
+  uint32_t c00, dd;
+  __device__ __forceinline__ void init(const uint16_t* __restrict__ cb_row) {
+    const uint32_t c = __ldg(reinterpret_cast<const uint32_t*>(cb_row));
+    c00 = prmt(c, c, 0x1010u);
+    dd = c00 ^ prmt(c, c, 0x3232u);
+  }
+  __device__ __forceinline__ uint32_t select(uint32_t v) const {
+    const uint32_t mask = prmt(v, v, 0xBB99u);
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x6C;" : "=r"(d) : "r"(mask), "r"(c00), "r"(dd));   // c00 ^ (mask & dd)
+    return d;
+  }
+};
+
 // Powers of two read from constant memory: a multiply by one of these is a left shift that issues on the
 // FMA pipe (IMAD) instead of the half-rate integer pipe that the decode saturates.
 static __constant__ uint32_t kPow2[16] = {1u << 0, 1u << 1, 1u << 2,  1u << 3,  1u << 4,  1u << 5,  1u << 6,  1u << 7,

@@ -20,6 +20,9 @@ KMQ_ERR_WORKSPACE, KMQ_ERR_LAYOUT, KMQ_ERR_CUDA = 5, 6, 7
 KMQ_ERR_SCRATCH_LIMIT = 8
 KMQ_LAYOUT_CANONICAL = 0
 KMQ_LAYOUT_TUNED = 1
+KMQ_LAYOUT_TABLE = 2
+KMQ_DEVICE_ERROR_WAIT_TIMEOUT = 1
+KMQ_DEVICE_ERROR_SMEM_WINDOW = 2
 
 _i64, _int, _ptr, _sz = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t
 
@@ -30,6 +33,8 @@ SIGNATURES = {
     "kmq_packed_bytes": (_sz, [_i64, _i64, _int, _int]),
     "kmq_packed_word_index": (_i64, [_i64, _i64, _i64, _i64, _int, _int]),
     "kmq_packed_field_shift": (_int, [_int, _int, _int]),
+    "kmq_packed_bit_index": (_i64, [_i64, _i64, _int, _i64, _i64, _int, _int]),
+    "kmq_preferred_layout": (_int, [_i64, _i64, _int, _i64]),
     "kmq_workspace_bytes": (_sz, [_i64, _i64, _int, _i64, _int]),
     "kmq_linear_num_launches": (_int, [_i64, _i64, _int, _i64, _int]),
     "kmq_linear_variant": (ctypes.c_char_p, [_i64, _i64, _int, _i64, _int]),
@@ -107,6 +112,14 @@ def kmq_packed_word_index(n, j, N, K, bits, layout=KMQ_LAYOUT_CANONICAL) -> int:
 
 def kmq_packed_field_shift(i, bits, layout=KMQ_LAYOUT_CANONICAL) -> int:
     return lib().kmq_packed_field_shift(i, bits, layout)
+
+
+def kmq_packed_bit_index(n, k, plane, N, K, bits, layout=KMQ_LAYOUT_CANONICAL) -> int:
+    return lib().kmq_packed_bit_index(n, k, plane, N, K, bits, layout)
+
+
+def kmq_preferred_layout(N, K, bits, M) -> int:
+    return lib().kmq_preferred_layout(N, K, bits, M)
 
 
 def kmq_workspace_bytes(N, K, bits, M, layout=KMQ_LAYOUT_CANONICAL) -> int:

@@ -100,3 +100,21 @@ def tuned_from_canonical(words: np.ndarray, bits: int) -> np.ndarray:
     j = np.arange(wpr)[None, :]
     out[(((n // 16) * steps + j // 16) * 16 + n % 16) * 16 + j % 16] = perm
     return out
+
+
+def table_from_indices(idx: np.ndarray, bits: int) -> np.ndarray:
+    """The documented bit-plane layout KMQ_LAYOUT_TABLE (include/kmq.h) applied to indices [N, K] (bits = 1, 2):
+    uint8 array of kmq_packed_bytes(..., TABLE) bytes, padding zero.  Written from the header's formulas."""
+    N, K = idx.shape
+    assert bits in (1, 2) and K % 8 == 0
+    chunks, tiles = -(-K // 256), -(-N // 16)
+    out = np.zeros(tiles * chunks * bits * 512, dtype=np.uint8)
+    n = np.arange(N)[:, None]
+    g = np.arange(K // 8)[None, :]
+    weights = (1 << np.arange(8)).astype(np.uint16)
+    for p in range(bits):
+        plane = ((idx.reshape(N, K // 8, 8) >> p) & 1).astype(np.uint16)
+        byte = (plane * weights).sum(axis=2).astype(np.uint8)                 # weight 8g + t in bit t
+        off = ((n // 16 * chunks + g // 32) * bits + p) * 512 + (2 * (n % 16) + g % 2) * 16 + ((g % 32) // 2 - n % 16) % 16
+        out[off] = byte
+    return out

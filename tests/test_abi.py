@@ -78,7 +78,7 @@ A = 0x1000  # a non-NULL, 16-byte aligned fake address; never dereferenced: vali
     (lambda: kmq.kmq_linear(A, A, A, A, 4, 32, 8, 1, stream=0, check=False), kmq.KMQ_ERR_BITS),
     (lambda: kmq.kmq_linear(A, A, A, A, 4, 32, 1, 0, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
     (lambda: kmq.kmq_linear(A, A, A, A, 4, 0, 1, 1, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
-    (lambda: kmq.kmq_linear(A, A, A, A, 4, 32, 1, 1, layout=2, stream=0, check=False), kmq.KMQ_ERR_LAYOUT),
+    (lambda: kmq.kmq_linear(A, A, A, A, 4, 32, 1, 1, layout=9, stream=0, check=False), kmq.KMQ_ERR_LAYOUT),
     (lambda: kmq.kmq_linear(A, A + 2, A, A, 4, 32, 1, 1, stream=0, check=False), kmq.KMQ_ERR_ALIGN),
     (lambda: kmq.kmq_linear_host(A, A, 0, A, 4, 32, 1, 1, A, A, stream=0, check=False), kmq.KMQ_ERR_NULL),
     (lambda: kmq.kmq_linear_host(A, A, A, A, 4, 32, 5, 1, A, A, stream=0, check=False), kmq.KMQ_ERR_BITS),

@@ -22,12 +22,13 @@ def random_layer(rng, N, K, bits, M):
     return idx, cb, x
 
 
-LAYOUTS = (kmq.KMQ_LAYOUT_CANONICAL, kmq.KMQ_LAYOUT_TUNED)
+LAYOUTS = (kmq.KMQ_LAYOUT_CANONICAL, kmq.KMQ_LAYOUT_TUNED, kmq.KMQ_LAYOUT_TABLE)
 
 
 def check_all(idx, cb, x, bits, what=""):
-    """Both packed layouts.  The canonical words must equal the oracle's bit for bit; the tuned words are defined
-    only through what they decode to (indices, weights), which must be exact, and their padding must be zero."""
+    """Every packed layout.  The canonical words must equal the oracle's bit for bit; the tuned and the table layout
+    are defined only through what they decode to (indices, weights), which must be exact; their bytes must also be
+    the documented arrangement of the oracle's indices, padding zero."""
     N, K = idx.shape
     ref_packed = orc.pack_canonical(idx, bits)
     ref_w = orc.dequant_bits(ref_packed, cb, K, bits)
@@ -40,8 +41,13 @@ def check_all(idx, cb, x, bits, what=""):
             assert np.array_equal(gu.packed_to_numpy(packed, N), ref_packed), f"{tag}: packed words differ"
         else:
             assert np.array_equal(gu.gpu_unpack(packed, N, K, bits, layout), idx), f"{tag}: unpack(pack(idx)) != idx"
-            assert np.array_equal(packed.cpu().numpy().view(np.uint32), gu.tuned_from_canonical(ref_packed, bits)), \
-                f"{tag}: tuned words differ from the documented layout"
+            if layout == kmq.KMQ_LAYOUT_TABLE and bits != 4:
+                assert np.array_equal(packed.cpu().numpy().view(np.uint8),
+                                      gu.table_from_indices(orc.unpack_canonical(ref_packed, K, bits), bits)), \
+                    f"{tag}: bit planes differ from the documented layout"
+            else:
+                assert np.array_equal(packed.cpu().numpy().view(np.uint32), gu.tuned_from_canonical(ref_packed, bits)), \
+                    f"{tag}: tuned words differ from the documented layout"
         w = gu.gpu_dequant(packed, cb, N, K, bits, layout)
         assert np.array_equal(w, ref_w), f"{tag}: dequantised weights differ"
         y = gu.gpu_linear(packed, cb, x, N, K, bits, layout)

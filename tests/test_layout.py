@@ -52,3 +52,44 @@ def test_field_shifts(bits):
     if bits == 1:
         assert tuned == [(31 - i // 2) if i % 2 else (15 - i // 2) for i in range(per)]
     assert kmq.kmq_packed_field_shift(per, bits, T) == -1 and kmq.kmq_packed_field_shift(0, 3, T) == -1
+
+
+@pytest.mark.parametrize("bits", (1, 2))
+@pytest.mark.parametrize("N,K", [(1, 32), (16, 256), (37, 544), (33, 288)])
+def test_table_layout_bit_index_is_injective_and_documented(bits, N, K):
+    """KMQ_LAYOUT_TABLE: every index bit has its own position inside kmq_packed_bytes, at the place the header's
+    formula gives; the word-based helpers do not describe this layout."""
+    L = kmq.KMQ_LAYOUT_TABLE
+    chunks, tiles = -(-K // 256), -(-N // 16)
+    total = kmq.kmq_packed_bytes(N, K, bits, L)
+    assert total == tiles * chunks * bits * 512
+    seen = set()
+    for n in range(N):
+        for k in range(K):
+            g = k // 8
+            for p in range(bits):
+                pos = kmq.kmq_packed_bit_index(n, k, p, N, K, bits, L)
+                byte = (((n // 16) * chunks + g // 32) * bits + p) * 512 + (2 * (n % 16) + g % 2) * 16 \
+                    + ((g % 32) // 2 - n % 16) % 16
+                assert pos == byte * 8 + k % 8
+                assert 0 <= pos < total * 8 and pos not in seen
+                seen.add(pos)
+    assert kmq.kmq_packed_word_index(0, 0, N, K, bits, L) == -1
+    assert kmq.kmq_packed_field_shift(0, bits, L) == -1
+    assert kmq.kmq_packed_bit_index(N, 0, 0, N, K, bits, L) == -1
+    assert kmq.kmq_packed_bit_index(0, K, 0, N, K, bits, L) == -1
+    assert kmq.kmq_packed_bit_index(0, 0, bits, N, K, bits, L) == -1
+
+
+@pytest.mark.parametrize("bits", (1, 2, 4))
+def test_bit_index_agrees_with_word_index_and_shift(bits):
+    N, K = 19, (32 // bits) * 5
+    per = 32 // bits
+    for layout in (C, T) + ((kmq.KMQ_LAYOUT_TABLE,) if bits == 4 else ()):
+        for n in (0, 7, 18):
+            for k in (0, 1, per - 1, per, K - 1):
+                w = kmq.kmq_packed_word_index(n, k // per, N, K, bits, layout)
+                sh = kmq.kmq_packed_field_shift(k % per, bits, layout)
+                for p in range(bits):
+                    assert kmq.kmq_packed_bit_index(n, k, p, N, K, bits, layout) == w * 32 + sh + p
+    assert kmq.kmq_packed_bytes(N, K, 4, kmq.KMQ_LAYOUT_TABLE) == kmq.kmq_packed_bytes(N, K, 4, T)
