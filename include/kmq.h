@@ -13,8 +13,11 @@
  * Conventions shared by every entry point
  *   - Pointers marked DEVICE are CUDA device pointers valid on the current
  *     device; HOST pointers are ordinary (ideally pinned) host memory.  The
- *     caller owns every buffer.  The library allocates no memory and keeps no
- *     state besides a per-device cache of device properties.
+ *     caller owns every buffer.  The library allocates no memory.  The state
+ *     it keeps per device: a cache of device properties and of a few symbol
+ *     addresses, two sticky error words in device memory (see
+ *     kmq_device_error_flags) and the fixed 512 KiB scratch array of
+ *     kmq_linear_static_scratch, which is part of the library image.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Work is enqueued on it and the call returns without synchronising,
  *     unless stated otherwise.
@@ -161,6 +164,12 @@ kmq_status kmq_unpack(const uint32_t* packed, int64_t N, int64_t K, int bits, in
  * The order of the fp32 summation is fixed for a given shape and device, so
  * repeated calls give bit-identical results.  Outputs for non-finite inputs
  * are unspecified.
+ * The return value covers validation and the launch itself.  The variants
+ * "tcgen05_*" and "table_*" (see kmq_linear_variant) wait on hardware
+ * barriers for asynchronous copies and matrix instructions; those waits are
+ * bounded, and one that runs out (which takes a GPU that has stopped
+ * delivering) leaves y incomplete and is reported only through
+ * kmq_device_error_flags(), which synchronises the device.
  */
 kmq_status kmq_linear(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x,
                       uint16_t* y, int64_t N, int64_t K, int bits, int64_t M, int layout,
@@ -229,10 +238,11 @@ kmq_status kmq_linear_tcgen05(const uint32_t* packed, const uint16_t* codebooks,
 
 /*
  * kmq_device_error_flags -- error word of the kernels on the current device.
- * The tensor-memory kernel behind kmq_linear_tcgen05 waits on hardware
- * barriers for its asynchronous matrix instructions; every such wait has an
- * iteration limit, and a warp whose wait runs out stops, stores nothing and
- * sets bit 0 here; the CTA still frees its tensor memory
+ * The tensor-memory kernel ("tcgen05_*" variants, kmq_linear_tcgen05) and the
+ * table kernel ("table_*" variants) wait on hardware barriers for asynchronous
+ * matrix instructions and bulk copies; every such wait gives up after 100 ms
+ * on the GPU's global timer, and a warp whose wait runs out stops, stores
+ * nothing more and sets bit 0 here; the CTA still frees its tensor memory
  * (the outputs of that call are then incomplete).  The call synchronises the
  * device, writes the word to *flags (host pointer) and clears it.  0 = no
  * kernel gave up since the last call.

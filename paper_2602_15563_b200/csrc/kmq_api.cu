@@ -136,19 +136,33 @@ kmq_status kmq_unpack(const uint32_t* packed, int64_t N, int64_t K, int bits, in
   return launch_unpack(packed, N, K, bits, layout, idx, (cudaStream_t)stream) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
 }
 
-kmq_status kmq_linear(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x, uint16_t* y, int64_t N,
-                      int64_t K, int bits, int64_t M, int layout, void* workspace, size_t workspace_bytes,
-                      void* stream) {
+namespace {
+
+// Every check of kmq_linear that needs no GPU work; on success `plan` is the kernel variant to launch.
+kmq_status check_linear_args(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x, const uint16_t* y,
+                             int64_t N, int64_t K, int bits, int64_t M, int layout, const void* workspace,
+                             size_t workspace_bytes, LinearPlan* plan) {
   if (!packed || !codebooks || !x || !y) return KMQ_ERR_NULL;
   if (kmq_status s = check_shape(N, K, bits, M)) return s;
   if (!known_layout(layout)) return KMQ_ERR_LAYOUT;
   if (!aligned16(packed) || !aligned16(codebooks) || !aligned16(x) || !aligned16(y)) return KMQ_ERR_ALIGN;
   if (!device_info()) return KMQ_ERR_CUDA;
-  const LinearPlan plan = plan_linear(N, K, bits, M, layout);
-  if (plan.workspace > 0) {
-    if (!workspace || workspace_bytes < plan.workspace) return KMQ_ERR_WORKSPACE;
+  *plan = plan_linear(N, K, bits, M, layout);
+  if (plan->workspace > 0) {
+    if (!workspace || workspace_bytes < plan->workspace) return KMQ_ERR_WORKSPACE;
     if (!aligned16(workspace)) return KMQ_ERR_ALIGN;
   }
+  return KMQ_OK;
+}
+
+}  // namespace
+
+kmq_status kmq_linear(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x, uint16_t* y, int64_t N,
+                      int64_t K, int bits, int64_t M, int layout, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+  LinearPlan plan;
+  if (kmq_status s = check_linear_args(packed, codebooks, x, y, N, K, bits, M, layout, workspace, workspace_bytes, &plan))
+    return s;
   return launch_linear(plan, packed, codebooks, x, y, N, K, bits, M, layout, workspace, (cudaStream_t)stream) ==
                  cudaSuccess
              ? KMQ_OK
@@ -158,14 +172,16 @@ kmq_status kmq_linear(const uint32_t* packed, const uint16_t* codebooks, const u
 kmq_status kmq_linear_host(const uint32_t* packed, const uint16_t* codebooks, const uint16_t* x_host, uint16_t* y_host,
                            int64_t N, int64_t K, int bits, int64_t M, int layout, uint16_t* x_dev, uint16_t* y_dev,
                            void* workspace, size_t workspace_bytes, void* stream) {
-  if (!x_host || !y_host || !x_dev || !y_dev) return KMQ_ERR_NULL;
-  if (!packed || !codebooks) return KMQ_ERR_NULL;
-  if (kmq_status s = check_shape(N, K, bits, M)) return s;
+  if (!x_host || !y_host) return KMQ_ERR_NULL;
+  // everything is validated before the first copy is enqueued: a failed check launches nothing
+  LinearPlan plan;
+  if (kmq_status s = check_linear_args(packed, codebooks, x_dev, y_dev, N, K, bits, M, layout, workspace,
+                                       workspace_bytes, &plan))
+    return s;
   cudaStream_t st = (cudaStream_t)stream;
   if (cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return KMQ_ERR_CUDA;
-  if (kmq_status s = kmq_linear(packed, codebooks, x_dev, y_dev, N, K, bits, M, layout, workspace, workspace_bytes,
-                                stream))
-    return s;
+  if (launch_linear(plan, packed, codebooks, x_dev, y_dev, N, K, bits, M, layout, workspace, st) != cudaSuccess)
+    return KMQ_ERR_CUDA;
   if (cudaMemcpyAsync(y_host, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KMQ_ERR_CUDA;
   return cudaStreamSynchronize(st) == cudaSuccess ? KMQ_OK : KMQ_ERR_CUDA;
 }

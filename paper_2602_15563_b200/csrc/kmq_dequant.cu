@@ -27,10 +27,15 @@ __device__ __forceinline__ uint4 decode8(uint32_t v, uint32_t c0, uint32_t c1, c
       o[p] = __byte_perm(c0, c1, 0x1010u + i0 * 0x22u + i1 * 0x2200u);
     }
   } else {
+    // c0 = this lane's share of the row's codebook: centroid (lane % 16) in the low half word.  A lookup is a
+    // shuffle from the lane that holds the entry (all 32 lanes of the warp must be here); two lookups are packed
+    // by one PRMT.  This keeps the 16 entries out of the load path, which the packed words and the stores need.
+    (void)row_cb;
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
       const uint32_t i0 = (v >> (8 * p)) & 15u, i1 = (v >> (8 * p + 4)) & 15u;
-      o[p] = (uint32_t)__ldg(row_cb + i0) | ((uint32_t)__ldg(row_cb + i1) << 16);
+      const uint32_t lo = __shfl_sync(0xFFFFFFFFu, c0, (int)i0), hi = __shfl_sync(0xFFFFFFFFu, c0, (int)i1);
+      o[p] = __byte_perm(lo, hi, 0x5410u);
     }
   }
   return make_uint4(o[0], o[1], o[2], o[3]);
@@ -45,6 +50,7 @@ __device__ __forceinline__ void load_codebook(const uint16_t* __restrict__ row_c
     c0 = cw.x;
     c1 = cw.y;
   }
+  if constexpr (BITS == 4) c0 = __ldg(row_cb + (threadIdx.x & 15));
 }
 
 // One CTA walks rows (grid-stride); inside a row every thread turns 8 weights into one 16-byte streaming store,
@@ -66,9 +72,14 @@ __global__ void __launch_bounds__(256) dequant_rows_kernel(const uint32_t* __res
     uint32_t c0, c1;
     load_codebook<BITS>(row_cb, c0, c1);
     uint4* out = reinterpret_cast<uint4*>(W + n * K);
-    for (int c = threadIdx.x; c < cpr; c += 256) {
-      uint32_t v;
-      if constexpr (TUNED) {
+    // b = 4 looks its centroids up by warp shuffles, so there whole warps stay in the loop (lanes past the end of
+    // the row decode a zero word and store nothing)
+    const int cend = BITS == 4 ? (cpr + 31) & ~31 : cpr;
+    for (int c = threadIdx.x; c < cend; c += 256) {
+      const bool live = BITS != 4 || c < cpr;
+      uint32_t v = 0;
+      if (!live) {
+      } else if constexpr (TUNED) {
         const int j = c / CPW, q = c % CPW;
         const uint32_t t = __ldg(row_words + (int64_t)(j >> 4) * 256 + (j & 15));
         if constexpr (BITS == 4) {
@@ -93,7 +104,8 @@ __global__ void __launch_bounds__(256) dequant_rows_kernel(const uint32_t* __res
       } else {
         v = __ldg(reinterpret_cast<const uint8_t*>(row_words) + c);
       }
-      stg_stream_u4(out + c, decode8<BITS>(v, c0, c1, row_cb));
+      const uint4 w8 = decode8<BITS>(v, c0, c1, row_cb);
+      if (live) stg_stream_u4(out + c, w8);
     }
   }
 }

@@ -37,7 +37,7 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
       const int64_t per = linear_multi_rows_per_launch(bits);
       p.variant = kVariantMulti;
       p.launches = (int)((M + per - 1) / per);
-      p.name = bits == 4 ? "multi_table_b4" : bits == 2 ? "multi_prmt_b2" : "multi_sign_b1";
+      p.name = bits == 4 ? "multi_table_b4" : bits == 2 ? "multi_prmt_b2" : "multi_select_b1";
       return p;
     }
     if (tuned) {
@@ -47,13 +47,13 @@ LinearPlan plan_linear(int64_t N, int64_t K, int bits, int64_t M, int layout) {
         p.launches = 2;
         p.split_k = ctas;
         p.workspace = linear_split_scratch_bytes(ctas);
-        p.name = bits == 4 ? "split_pairtable_b4" : bits == 2 ? "split_prmt_b2" : "split_sign_b1";
+        p.name = bits == 4 ? "split_pairtable_b4" : bits == 2 ? "split_prmt_b2" : "split_select_b1";
         return p;
       }
     }
     if (bits == 4) p.name = tuned ? "tiled_pairtable_b4" : "staged_pairtable_b4";
     else if (bits == 2) p.name = tuned ? "tiled_prmt_b2" : "staged_prmt_b2";
-    else p.name = tuned ? "tiled_sign_b1" : "staged_sign_b1";
+    else p.name = tuned ? "tiled_select_b1" : "staged_select_b1";
   } else {
     p.variant = kVariantGeneric;
     p.launches = 1;

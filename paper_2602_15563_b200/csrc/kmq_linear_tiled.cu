@@ -1,5 +1,5 @@
-// kmq_linear on the tuned (tile-major) packed layout, small batches (M <= 8; larger ones and, at b = 1, M >= 4 go
-// to the multi-tile kernel).
+// kmq_linear on the tuned (tile-major) packed layout, small batches (M <= 8; larger ones, and from
+// linear_multi_min_rows() batch rows on also smaller ones, go to the multi-tile kernel).
 //
 // One CTA owns one tile of 16 output rows; its 8 warps split K step by step (a step = 64 packed bytes of each
 // row = 1 KB of the tile, stored contiguously).  Per step a warp
@@ -22,23 +22,12 @@
 namespace kmq {
 namespace {
 
-#ifndef KMQ_TILED_WARPS
-#define KMQ_TILED_WARPS 8
-#endif
-#ifndef KMQ_TILED_MINB
-#define KMQ_TILED_MINB 3
-#endif
-#ifndef KMQ_TILED_STAGES4
-#define KMQ_TILED_STAGES4 2
-#endif
-constexpr int kWarps = KMQ_TILED_WARPS;
+constexpr int kWarps = 8;
+constexpr int kMinCtasPerSm = 3;   // register budget of the launch bounds
 constexpr int kThreads = kWarps * 32;
 constexpr int kRows = kTileRows;
 constexpr int kPairEntryStride = 256;   // b = 4 tables: entry e, half h, lane l at e * 256 + h * 128 + l * 4
 constexpr int kTableBytes4 = 256 * kPairEntryStride;
-#ifndef KMQ_PDL
-#define KMQ_PDL 1
-#endif
 
 template <int BITS>
 struct TGeo {
@@ -50,7 +39,7 @@ struct TGeo {
   static constexpr int kRowStride = 4 * kChunkStride;     // one batch row of one step
   static constexpr int kPiecesPerRow = kStepK / 8;        // 16-byte pieces of x per batch row and step
   static constexpr int kTableBytes = BITS == 4 ? kTableBytes4 : 0;
-  static constexpr int kStages = BITS == 4 ? KMQ_TILED_STAGES4 : 2;       // steps in flight per warp (deeper rings measured slower)
+  static constexpr int kStages = 2;                       // steps in flight per warp (deeper rings measured slower)
 };
 
 template <int BITS, int MMAX>
@@ -258,24 +247,20 @@ __device__ __forceinline__ void store_output(float v, uint16_t* __restrict__ y, 
 
 // One CTA per tile.
 template <int BITS, int MMAX>
-__global__ void __launch_bounds__(kThreads, KMQ_TILED_MINB) linear_tiled_kernel(const uint32_t* __restrict__ packed,
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm) linear_tiled_kernel(const uint32_t* __restrict__ packed,
                                                                     const uint16_t* __restrict__ cb,
                                                                     const uint16_t* __restrict__ x,
                                                                     uint16_t* __restrict__ y, int64_t N, int64_t K,
                                                                     int M) {
-#if KMQ_PDL
   // Programmatic dependent launch: nothing is read before the previous kernel on the stream has completed (same
   // ordering as a plain launch), but this grid could be set up while that kernel drained, and the next kernel may be
   // set up while this one sums and stores.
   asm volatile("griddepcontrol.wait;" ::: "memory");
-#endif
   const int steps = (int)((K / (4 * TGeo<BITS>::kWordK) + 3) >> 2);
   const int64_t row0 = (int64_t)blockIdx.x * kRows;
   float v;
   tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, blockIdx.x, 0, steps, v);
-#if KMQ_PDL
   asm volatile("griddepcontrol.launch_dependents;");
-#endif
   store_output(v, y, N, M, row0);
 }
 
@@ -289,7 +274,7 @@ __global__ void __launch_bounds__(kThreads, KMQ_TILED_MINB) linear_tiled_kernel(
 constexpr int kSlotFloats = kRows * 8 + 8;   // 128 sums (+ 8 unused: keeps the slots 32-byte aligned)
 
 template <int BITS, int MMAX>
-__global__ void __launch_bounds__(kThreads, KMQ_TILED_MINB) linear_split_kernel(const uint32_t* __restrict__ packed,
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm) linear_split_kernel(const uint32_t* __restrict__ packed,
                                                                     const uint16_t* __restrict__ cb,
                                                                     const uint16_t* __restrict__ x,
                                                                     uint16_t* __restrict__ y, int64_t N, int64_t K,
@@ -350,7 +335,7 @@ cudaError_t launch_one(const uint32_t* packed, const uint16_t* cb, const uint16_
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = KMQ_PDL ? 1 : 0;
+  cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, linear_tiled_kernel<BITS, MMAX>, packed, cb, x, y, N, K, M);
 }
 
@@ -422,15 +407,45 @@ namespace kmq {
 // Every range restarts the load pipeline and the decode set-up once or twice more than a whole tile would, so this
 // only pays when a tile is long: at least kSplitMinSteps steps (measured: 8192 x 28672, b = 4, 224 steps, 55 -> 44 us;
 // with 16..56 steps per tile the per-tile grid is faster).
-#ifndef KMQ_SPLIT_MIN_STEPS
-#define KMQ_SPLIT_MIN_STEPS 128
-#endif
-constexpr int64_t kSplitMinSteps = KMQ_SPLIT_MIN_STEPS;
+constexpr int64_t kSplitMinSteps = 128;
+
+namespace {
+
+// CTAs of linear_split_kernel<BITS, MMAX> that fit one SM (registers and shared memory), asked from the runtime
+// once per device and instantiation.
+template <int BITS, int MMAX>
+int split_ctas_per_sm() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  if (cached[dev] == 0) {
+    constexpr int smem = TSmem<BITS, MMAX>::kTotal;
+    int n = 0;
+    if (cudaFuncSetAttribute(linear_split_kernel<BITS, MMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+            cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, linear_split_kernel<BITS, MMAX>, kThreads, smem) !=
+            cudaSuccess)
+      return 0;
+    cached[dev] = n > 0 ? n : -1;
+  }
+  return cached[dev] > 0 ? cached[dev] : 0;
+}
+
+template <int BITS>
+int split_ctas_per_sm_bits(int64_t M) {
+  return M == 1 ? split_ctas_per_sm<BITS, 1>() : M == 2 ? split_ctas_per_sm<BITS, 2>() : split_ctas_per_sm<BITS, 4>();
+}
+
+}  // namespace
 
 int linear_split_ctas(int64_t N, int64_t K, int bits, int64_t M) {
   const DeviceInfo* di = device_info();
-  if (!di || M >= linear_multi_min_rows(bits, N)) return 0;
-  const int64_t slots = (int64_t)di->sm_count * 3;
+  if (!di || M > 4 || M >= linear_multi_min_rows(bits, N)) return 0;
+  // one CTA per resident slot of the instantiation that will run, so that there is no second wave
+  const int per_sm = bits == 1 ? split_ctas_per_sm_bits<1>(M) : bits == 2 ? split_ctas_per_sm_bits<2>(M)
+                                                                            : split_ctas_per_sm_bits<4>(M);
+  if (per_sm <= 0) return 0;
+  const int64_t slots = (int64_t)di->sm_count * per_sm;
   const int64_t tiles = (N + kRows - 1) / kRows;
   const int64_t steps = (K * bits / 128 + 3) / 4;
   return (tiles > slots && steps >= kSplitMinSteps) ? (int)slots : 0;

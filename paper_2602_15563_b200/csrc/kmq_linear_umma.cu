@@ -48,14 +48,11 @@ template <int NB>
 constexpr int ring_depth() {
   return NB > 64 ? 4 : 6;
 }
-#ifndef KMQ_UMMA_WRING
-#define KMQ_UMMA_WRING 6
-#endif
-constexpr int kWRing = KMQ_UMMA_WRING;                   // ring of 1 KB steps of packed words per tile (cp.async), kWRing - 1 in flight
+constexpr int kWRing = 6;                   // ring of 1 KB steps of packed words per tile (cp.async), kWRing - 1 in flight
 constexpr int kWRowStride = 80;                          // a row's 64 bytes of a step, padded: lanes read consecutive rows
 constexpr int kWStepBytes = kBM * kWRowStride;
 constexpr uint32_t kWaitHintNs = 20000;                  // one try_wait on an mbarrier may park the thread this long
-constexpr uint32_t kWaitLimit = 1u << 12;                // tries before giving up (at most about 80 ms)
+constexpr uint64_t kWaitLimitNs = 100ull * 1000 * 1000;  // a wait gives up after this much time on the global timer
 
 template <int BITS>
 struct UGeo {
@@ -179,9 +176,11 @@ __device__ __forceinline__ void load_acc(uint32_t (&w)[NC], uint32_t taddr, bool
 }
 
 // Bounded wait for the phase of parity `parity` of an mbarrier.  try_wait parks the thread in hardware for up to the
-// hinted time instead of spinning, so waiting warps do not take issue slots from the ones that decode.
+// hinted time instead of spinning, so waiting warps do not take issue slots from the ones that decode.  The hint is
+// only a hint (a try may come back early), so the bound is taken on the global timer, not on the number of tries.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+  uint64_t t0 = 0;
+  for (;;) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.b32 %0, 1, 0, p;\n\t}"
@@ -189,8 +188,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         : "r"(bar), "r"(parity), "r"(kWaitHintNs)
         : "memory");
     if (done) return true;
+    uint64_t now;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+    if (t0 == 0) t0 = now;
+    else if (now - t0 > kWaitLimitNs) return false;
   }
-  return false;
 }
 
 // Decode state of a thread's output row.
@@ -497,6 +499,10 @@ __global__ void __launch_bounds__(kThreads, 1) linear_umma_kernel(const uint32_t
   }
   tc_fence_before_sync();
   __syncthreads();
+  // The tensor memory is given back on every path, also after a wait ran out: a CTA that left without freeing its
+  // columns would block every later CTA on this SM in tcgen05.alloc for good.  A wait only runs out after 100 ms,
+  // five orders of magnitude beyond the life of any instruction this kernel issues, so nothing of this CTA can
+  // still be using the columns then.
   if (warp == kDecodeWarps)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)SM::kTmemCols)
                  : "memory");
@@ -538,10 +544,24 @@ bool make_x_map(CUtensorMap* map, const uint16_t* x, int64_t K, int M) {
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Dynamic shared memory to launch with: what the kernel uses, but more than half of what an SM offers (the opt-in
+// maximum per CTA is the SM's shared memory minus the 1 KB the system keeps per CTA).
+inline int umma_launch_smem(int kernel_bytes, int max_smem_optin) {
+  const int more_than_half = max_smem_optin / 2 + 1024;
+  return kernel_bytes > more_than_half ? kernel_bytes : more_than_half;
+}
+
 template <int BITS, int NB>
 cudaError_t launch_nb(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N, int64_t K,
                       int M, cudaStream_t s) {
-  constexpr int smem = USmem<BITS, NB>::kTotal;
+  // Every CTA takes all 512 tensor-memory columns with a blocking tcgen05.alloc and frees them only at its end, after
+  // cluster barriers: two such CTAs on one SM (of one cluster or of two) could wait for each other for ever.  The
+  // launch therefore asks for more than half of the SM's shared memory whatever the kernel needs, so that a second
+  // CTA can never become resident on the same SM.
+  const DeviceInfo* di = device_info();
+  if (!di) return cudaErrorInvalidDevice;
+  const int smem = umma_launch_smem(USmem<BITS, NB>::kTotal, di->max_smem_optin);
+  if (smem > di->max_smem_optin || 2 * (smem + 1024) <= di->max_smem_optin + 1024) return cudaErrorInvalidConfiguration;
   static bool configured[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);

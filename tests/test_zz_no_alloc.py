@@ -1,6 +1,7 @@
 """kmq_linear_static_scratch, the entry point for callers that may not allocate device memory (its scratch is a fixed
 array inside the library): on a shape that really uses scratch it must give what kmq_linear gives with a
-caller-provided workspace, on two calls in a row that share the array.  Collected last on purpose."""
+caller-provided workspace, on two calls in a row that share the array.  The file name sorts last on purpose: with
+`pytest -x` a failure here cannot keep any other test from running."""
 import numpy as np
 import pytest
 import torch
