@@ -46,6 +46,9 @@ WORKLOADS = {
     "config5": [("down_large", 8192, 28672, "laplace", b, m) for b in (1, 4) for m in (1, 16)] +
                [("down_large", 8192, 28672, "laplace", b, 0) for b in (1, 4)],     # M = 0: kmq_dequant_to_bf16
     "tiny": [("tiny", 256, 256, "normal", b, 1) for b in (1, 2, 4)],
+    # the larger batch-1 shapes of configurations 4 and 5 with random indices (no k-means fit: set-up in seconds)
+    "large": [("square8192", 8192, 8192, "random", 2, 1), ("down_large", 8192, 28672, "random", 1, 1),
+              ("down_large", 8192, 28672, "random", 4, 1)],
 }
 WORKLOAD_TEXT = {
     "config2": "single square layer N=K=4096, batch 1, b in {1,2,4}, per-row 2^b-centroid bf16 codebooks "
@@ -57,13 +60,15 @@ WORKLOAD_TEXT = {
     "config5": "large down projection N=8192 K=28672, b in {1,4}, batch in {1,16}, Laplace weights, plus the "
                "standalone kmq_dequant_to_bf16 of the full matrix (cases with M=0)",
     "tiny": "256x256 correctness layer",
+    "large": "batch-1 shapes of configurations 4 and 5 (8192x8192 b=2; 8192x28672 b=1, 4) with uniformly random "
+             "indices and sorted N(0, 0.02) codebooks: timing does not depend on the weight values",
 }
-CONFIG_ID = {"config2": 2, "config3_m1": 3, "config3_m8": 3, "config4": 4, "config5": 5, "tiny": 1}
+CONFIG_ID = {"config2": 2, "config3_m1": 3, "config3_m8": 3, "config4": 4, "config5": 5, "tiny": 1, "large": 90}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel,
-# from the ncu capture summarised under profiles/ (None = not captured yet).
-NCU_TRAFFIC_BYTES = {                      # (workload, bits, M) -> bytes; profiles/kmq_linear_tiled_config2_ncu_full.md
-    ("config2", 1, 1): 2141184, ("config2", 2, 1): 4249088, ("config2", 4, 1): 8539392,
+# dram__bytes_read.sum + dram__bytes_write.sum per call (all launches of the call) from the ncu captures summarised
+# under profiles/, keyed by (N, K, bits, M, variant); a case without an entry, or whose kernel has changed since the
+# capture, reports null.
+NCU_TRAFFIC_BYTES = {
 }
 
 
@@ -164,17 +169,32 @@ class ClockSampler(threading.Thread):
 class Case:
     """One (layer, bits, M) of the workload with its pool of device buffers."""
 
-    def __init__(self, name, N, K, dist, bits, M, config_id, torch, kmq, synth, pool_bytes, layout="auto"):
+    def __init__(self, name, N, K, dist, bits, M, config_id, torch, kmq, synth, pool_bytes, layout="auto",
+                 random_weights=False):
         self.name, self.N, self.K, self.bits, self.M = name, N, K, bits, M
         self.bytes = algorithmic_bytes(N, K, bits, M)
         self.pool = max(4, -(-pool_bytes // self.bytes))
-        layer = dict(cached_layer(synth, N, K, bits, dist, config_id))
         self.dequant = M == 0
+        self.random_weights = random_weights
         rng = synth.rng_for(config_id, 100 + bits * 1000 + M)
-        layer["x"] = synth.draw_activations(max(M, 1), K, synth.rng_for(config_id, synth.TENSOR_X))
-        self.layer = layer
+        x0 = synth.draw_activations(max(M, 1), K, synth.rng_for(config_id, synth.TENSOR_X))
         dev = torch.device("cuda")
-        idx = torch.from_numpy(layer["idx"]).to(dev)
+        if random_weights:
+            # timing does not depend on the weight values: uniformly random indices and sorted N(0, 0.02) codebooks,
+            # drawn on the GPU, spare the minutes a k-means fit of a 235 M-weight layer takes on the host
+            g = torch.Generator(device=dev).manual_seed(1000 * config_id + 10 * bits + M)
+            idx = torch.randint(0, 1 << bits, (N, K), dtype=torch.uint8, device=dev, generator=g)
+            cb_f = (torch.randn(N, 1 << bits, device=dev, generator=g) * 0.02).sort(dim=1).values
+            codebooks = cb_f.to(torch.bfloat16).view(torch.int16).cpu().numpy().view(np.uint16)
+        else:
+            layer = cached_layer(synth, N, K, bits, dist, config_id)
+            idx = torch.from_numpy(layer["idx"]).to(dev)
+            codebooks = layer["codebooks"]
+        # rows whose outputs the parity spot check recomputes with the oracle
+        self.check_rows = np.unique(np.concatenate([np.arange(16), np.arange(N - 16, N),
+                                                    np.random.default_rng(bits + M).choice(N, 32, replace=False)]))
+        self.check_idx = idx[torch.from_numpy(self.check_rows).to(dev)].cpu().numpy()
+        self.check_cb = codebooks[self.check_rows]
         # the layout in which the library is fastest for this batch (packing is the offline step)
         self.layout = {"tuned": kmq.KMQ_LAYOUT_TUNED, "table": kmq.KMQ_LAYOUT_TABLE,
                        "canonical": kmq.KMQ_LAYOUT_CANONICAL}.get(layout)
@@ -189,10 +209,10 @@ class Case:
         kmq.kmq_pack(idx, N, K, bits, self.packed[0], layout=self.layout)   # a1: offline packing, on the GPU
         self.packed[1:] = self.packed[0]
         del idx
-        cb = torch.from_numpy(layer["codebooks"].view(np.int16)).to(dev)
+        cb = torch.from_numpy(codebooks.view(np.int16)).to(dev)
         self.cb = cb.unsqueeze(0).repeat(self.pool, 1, 1).contiguous()
         Mx = max(M, 1)
-        xs = np.stack([layer["x"]] + [synth.draw_activations(Mx, K, rng) for _ in range(self.pool - 1)])
+        xs = np.stack([x0] + [synth.draw_activations(Mx, K, rng) for _ in range(self.pool - 1)])
         self.x_host = torch.from_numpy(xs.view(np.int16)).pin_memory()
         self.x = self.x_host.to(dev)
         if self.dequant:
@@ -221,6 +241,48 @@ class Case:
                                  layout=self.layout)
 
 
+def machine_probes(torch, kmq, stream):
+    """The two figures every per-call time is read against: the fixed cost of a call (a do-nothing kernel of the
+    library in the same graph-replay protocol) and the read-only streaming bandwidth of a kernel of the library."""
+    with torch.cuda.stream(stream):
+        kmq.kmq_probe_launch()
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(200):
+                kmq.kmq_probe_launch()
+        for _ in range(3):
+            g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(20):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+        floor_us = e0.elapsed_time(e1) * 1e3 / (20 * 200)
+        nbytes = 1 << 30
+        buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        buf.random_(0, 256)
+        out = torch.empty(kmq.kmq_probe_read_out_bytes(), dtype=torch.uint8, device="cuda")
+        best = float("inf")
+        for _ in range(6):
+            e0.record(stream)
+            kmq.kmq_probe_read(buf, nbytes, out)
+            e1.record(stream)
+            stream.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        del buf
+    return {"launch_floor_us": round(floor_us, 3),
+            "launch_floor_how": "do-nothing kernel of the library, 200 per CUDA graph, programmatic dependent launch",
+            "read_only_gbs": round(nbytes / (best * 1e-3) / 1e9, 1),
+            "read_only_how": "1 GiB read once with 128-bit streaming loads, best of 6"}
+
+
+# Cases timed next to the workload of --workload config2 (not part of `value`): shapes long enough for a steady-state
+# HBM fraction.  (layer name, N, K, bits, M)
+EXTRA_CASES = [(n, N, K, b, M) for (n, N, K, _d, b, M) in WORKLOADS["large"]]
+
+
 def run_library(args):
     import torch
     from paper_2602_15563_b200 import build as kb
@@ -245,8 +307,12 @@ def run_library(args):
     peak_gbs, peak_kind = measured_peak()
     cfg_id = CONFIG_ID[args.workload]
     pool_bytes = 2 * L2_BYTES
-    cases = [Case(n, N, K, d, b, M, cfg_id, torch, kmq, synth, pool_bytes, args.layout)
+    cases = [Case(n, N, K, d, b, M, cfg_id, torch, kmq, synth, pool_bytes, args.layout, random_weights=(d == "random"))
              for (n, N, K, d, b, M) in select_cases(args)]
+    n_main = len(cases)
+    if args.workload == "config2" and not args.case and not args.no_extra:
+        cases += [Case(n, N, K, "normal", b, M, 90, torch, kmq, synth, pool_bytes, args.layout, random_weights=True)
+                  for (n, N, K, b, M) in EXTRA_CASES]
 
     stream = torch.cuda.Stream()
     graphs = []
@@ -261,11 +327,13 @@ def run_library(args):
                     c.call(i)
             graphs.append(g)
 
-    def one_step(events=None):
-        for j, g in enumerate(graphs):
+    def one_step(events=None, lo=0, hi=None):
+        """One pass over the cases lo .. hi-1 (default: the workload itself, without the extra cases)."""
+        hi = n_main if hi is None else hi
+        for j in range(lo, hi):
             if events is not None:
                 events[j][0].record(stream)
-            g.replay()
+            graphs[j].replay()
             if events is not None:
                 events[j][1].record(stream)
 
@@ -292,15 +360,23 @@ def run_library(args):
             one_step(ev[s])
         t1.record(stream)
         barrier()
+        # ---- after the timed region: the extra cases, the same number of steps, their own events ----
+        if len(cases) > n_main:
+            for _ in range(3):
+                one_step(None, n_main, len(cases))
+            for s in range(args.steps):
+                one_step(ev[s], n_main, len(cases))
+            barrier()
         sampler.active = False
+        machine = machine_probes(torch, kmq, stream) if rank == 0 and not args.quick else None
     elapsed_ms = t0.elapsed_time(t1)
     step_ms = [[ev[s][j][0].elapsed_time(ev[s][j][1]) for s in range(args.steps)] for j in range(len(cases))]
     per_case_ms = [sum(t) / args.steps for t in step_ms]
     # standard error of the mean per-call time over the K timed steps (each step = one replay of the case's graph)
     per_case_sem_ms = [(float(np.std(t, ddof=1)) / np.sqrt(len(t)) if len(t) > 1 else 0.0) for t in step_ms]
 
-    step_bytes = sum(c.bytes * c.pool for c in cases)
-    step_calls = sum(c.pool for c in cases)
+    step_bytes = sum(c.bytes * c.pool for c in cases[:n_main])
+    step_calls = sum(c.pool for c in cases[:n_main])
     if dist is not None:
         t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -319,12 +395,12 @@ def run_library(args):
             dist.destroy_process_group()
         return
     with torch.cuda.stream(stream):
-        for c in cases:
+        for c in cases[:n_main]:
             c.call_host(0)
         barrier()
         w0 = time.perf_counter()
         for _ in range(e2e_steps):
-            for c in cases:
+            for c in cases[:n_main]:
                 for i in range(c.pool):
                     c.call_host(i)
         torch.cuda.synchronize()
@@ -334,8 +410,8 @@ def run_library(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_s = float(t.item())
     e2e_value = world * step_bytes * e2e_steps / e2e_s / 1e9
-    h2d = sum(c.M * c.K * 2 * c.pool for c in cases)
-    d2h = sum(c.M * c.N * 2 * c.pool for c in cases)
+    h2d = sum(c.M * c.K * 2 * c.pool for c in cases[:n_main])
+    d2h = sum(c.M * c.N * 2 * c.pool for c in cases[:n_main])
 
     sampler.stop_flag = True
     sampler.join(timeout=1.0)
@@ -348,11 +424,10 @@ def run_library(args):
     from oracle import kmq_oracle as orc
     worst = 0.0
     checked = 0
-    for c in cases:
-        rows = np.unique(np.concatenate([np.arange(16), np.arange(c.N - 16, c.N),
-                                         np.random.default_rng(c.bits + c.M).choice(c.N, 32, replace=False)]))
-        ref_packed = orc.pack_canonical(c.layer["idx"][rows], c.bits)
-        cb_rows = c.layer["codebooks"][rows]
+    for ci, c in enumerate(cases):
+        rows = c.check_rows
+        ref_packed = orc.pack_canonical(c.check_idx, c.bits)
+        cb_rows = c.check_cb
         d_rows = torch.from_numpy(rows).cuda()
         for i in sorted({0, c.pool - 1}):
             if c.dequant:
@@ -363,28 +438,40 @@ def run_library(args):
                 x_i = c.x_host[i].numpy().view(np.uint16)
                 y_ref, s = orc.linear_f64(ref_packed, cb_rows, x_i, c.K, c.bits)
                 y = c.y[i][:, d_rows].cpu().numpy().view(np.uint16)
-                yh = c.y_host[i].numpy().view(np.uint16)[:, rows]
-                worst = max(worst, orc.check_linear(y, y_ref, s), orc.check_linear(yh, y_ref, s))
+                worst = max(worst, orc.check_linear(y, y_ref, s))
+                if ci < n_main:                  # the end-to-end leg ran on the workload's own cases
+                    yh = c.y_host[i].numpy().view(np.uint16)[:, rows]
+                    worst = max(worst, orc.check_linear(yh, y_ref, s))
             checked += 1
 
     # ---- per-case figures and the roofline of the dominant kernel ----
     per_case = []
-    for c, ms, sem in zip(cases, per_case_ms, per_case_sem_ms):
+    floor_us = machine["launch_floor_us"] if machine else None
+    for ci, (c, ms, sem) in enumerate(zip(cases, per_case_ms, per_case_sem_ms)):
         us = ms * 1e3 / c.pool
         gbs = c.bytes / (us * 1e-6) / 1e9
+        ideal_us = c.bytes / (peak_gbs * 1e9) * 1e6
         per_case.append({"layer": c.name, "N": c.N, "K": c.K, "bits": c.bits, "M": c.M, "pool": c.pool,
-                         "variant": c.variant, "layout": c.layout_name, "us_per_call": round(us, 3),
-                         "us_per_call_sem": round(sem * 1e3 / c.pool, 4), "gbs": round(gbs, 1),
-                         "frac_of_measured_hbm": round(gbs / peak_gbs, 4), "frac_of_8tbs": round(gbs / 8000.0, 4),
-                         "bytes_per_call": c.bytes})
-    dom = max(range(len(cases)), key=lambda j: per_case_ms[j])
+                         "variant": c.variant, "layout": c.layout_name, "launches_per_call": c.launches,
+                         "us_per_call": round(us, 3), "us_per_call_sem": round(sem * 1e3 / c.pool, 4),
+                         "gbs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peak_gbs, 4),
+                         "frac_of_8tbs": round(gbs / 8000.0, 4), "bytes_per_call": c.bytes,
+                         "ideal_us_at_measured_hbm": round(ideal_us, 3), "launch_floor_us": floor_us,
+                         "in_value": ci < n_main,
+                         "weights": "random indices, timing only" if c.random_weights else "k-means fit"})
+    # the kernel with the largest share of the step: achieved = algorithmic bytes of one call / time of one call
+    # (a call of two launches still moves its bytes once)
+    dom = max(range(n_main), key=lambda j: per_case_ms[j])
     dc = cases[dom]
-    achieved = per_case[dom]["gbs"] / dc.launches if dc.launches > 1 else per_case[dom]["gbs"]
+    achieved = per_case[dom]["gbs"]
     roofline = {"bound": "hbm", "kernel": f"kmq_linear[{dc.variant}] b={dc.bits} M={dc.M} {dc.N}x{dc.K}",
                 "achieved": round(achieved, 1), "peak": peak_gbs, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": round(achieved / peak_gbs, 4),
-                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dc.bits, dc.M)),
-                "algorithmic_bytes_per_launch": dc.bytes}
+                "traffic": NCU_TRAFFIC_BYTES.get((dc.N, dc.K, dc.bits, dc.M, dc.variant)),
+                "algorithmic_bytes_per_launch": dc.bytes,
+                "share_of_step": round(per_case_ms[dom] / sum(per_case_ms[:n_main]), 3)}
+    for row, c in zip(per_case, cases):
+        row["ncu_dram_bytes"] = NCU_TRAFFIC_BYTES.get((c.N, c.K, c.bits, c.M, c.variant))
 
     cpu = cpu_baseline(args.workload, budget_s=args.cpu_seconds)
 
@@ -406,7 +493,8 @@ def run_library(args):
         "cpu_baseline": cpu,
         "e2e": {"value": round(e2e_value, 2), "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "api": "kmq_linear_host (x from pinned host memory, y back to host, per call)"},
-        "gpu_launches": args.steps * sum(c.pool * c.launches for c in cases),
+        "gpu_launches": args.steps * sum(c.pool * c.launches for c in cases[:n_main]),
+        "machine": machine,
         "clocks": sampler.summary(),
         "parity": {"calls_checked": checked, "max_err_over_tol": round(worst, 4), "ok": bool(worst <= 1.0)},
         "paper_context": PAPER_CONTEXT,
@@ -448,11 +536,16 @@ def _oracle_cases(workload):
     from paper_2602_15563_b200 import synth
     out = []
     for (name, N, K, d, b, M) in WORKLOADS[workload]:
-        layer = cached_layer(synth, N, K, b, d, CONFIG_ID[workload])
         n = int(min(N, max(16, ORACLE_MAX_WEIGHTS // K)))
+        if d == "random":
+            rng = np.random.default_rng(1000 * CONFIG_ID[workload] + 10 * b + M)
+            idx = rng.integers(0, 1 << b, size=(n, K), dtype=np.uint8)
+            cbs = synth.f32_to_bf16_bits(np.sort(rng.standard_normal((n, 1 << b)) * 0.02, axis=1).astype(np.float32))
+        else:
+            layer = cached_layer(synth, N, K, b, d, CONFIG_ID[workload])
+            idx, cbs = layer["idx"][:n], layer["codebooks"][:n]
         x = synth.draw_activations(max(M, 1), K, synth.rng_for(CONFIG_ID[workload], synth.TENSOR_X))
-        out.append((n, K, b, M, orc.pack_canonical(layer["idx"][:n], b), layer["codebooks"][:n], x,
-                    algorithmic_bytes(n, K, b, M)))
+        out.append((n, K, b, M, orc.pack_canonical(idx, b), cbs, x, algorithmic_bytes(n, K, b, M)))
     return out
 
 
@@ -538,6 +631,8 @@ def main():
     ap.add_argument("--case", default="", help='subset of the workload, e.g. "bits=1,M=1" (keys: layer, N, K, bits, M)')
     ap.add_argument("--layout", default="auto", choices=["auto", "tuned", "table", "canonical"],
                     help="packed layout of the weights (auto = kmq_preferred_layout per case)")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="config2 only: skip the three larger cases timed next to the workload (outside `value`)")
     ap.add_argument("--quick", action="store_true",
                     help="kernel timing only (no end-to-end leg, CPU baseline or parity check): for profiler runs")
     args = ap.parse_args()

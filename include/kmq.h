@@ -263,6 +263,25 @@ kmq_status kmq_device_error_flags(unsigned int* flags);
 kmq_status kmq_dequant_to_bf16(const uint32_t* packed, const uint16_t* codebooks, uint16_t* W,
                                int64_t N, int64_t K, int bits, int layout, void* stream);
 
+/*
+ * Measurement helpers (conveniences of this library; the paper has no
+ * counterpart).  They put the layer's timings into proportion on the GPU at
+ * hand:
+ * kmq_probe_launch -- enqueue a kernel that does nothing, launched exactly as
+ *   the layer's kernels are (programmatic dependent launch): timing a chain of
+ *   these gives the fixed cost of a call, the floor under every layer whose
+ *   ideal time is a microsecond or two.
+ * kmq_probe_read -- read `bytes` (a multiple of 16) of DEVICE memory `buf`
+ *   once with 128-bit streaming loads and fold them into `out` (DEVICE,
+ *   kmq_probe_read_out_bytes() bytes): bytes / time is the read-only bandwidth
+ *   a kernel of this library can reach, the ceiling next to the copy
+ *   bandwidth that roofline fractions are quoted against.
+ * Errors: KMQ_ERR_NULL, KMQ_ERR_ALIGN, KMQ_ERR_CUDA.
+ */
+kmq_status kmq_probe_launch(void* stream);
+size_t kmq_probe_read_out_bytes(void);
+kmq_status kmq_probe_read(const void* buf, size_t bytes, void* out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

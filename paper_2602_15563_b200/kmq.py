@@ -47,6 +47,9 @@ SIGNATURES = {
     "kmq_linear_tcgen05": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _ptr]),
     "kmq_device_error_flags": (_int, [_ptr]),
     "kmq_dequant_to_bf16": (_int, [_ptr, _ptr, _ptr, _i64, _i64, _int, _int, _ptr]),
+    "kmq_probe_launch": (_int, [_ptr]),
+    "kmq_probe_read_out_bytes": (_sz, []),
+    "kmq_probe_read": (_int, [_ptr, _sz, _ptr, _ptr]),
 }
 
 
@@ -203,4 +206,24 @@ def kmq_dequant_to_bf16(packed, codebooks, W, N, K, bits, layout=KMQ_LAYOUT_CANO
     st = lib().kmq_dequant_to_bf16(_addr(packed), _addr(codebooks), _addr(W), N, K, bits, layout, _stream(stream))
     if check:
         _check(st, "kmq_dequant_to_bf16")
+    return st
+
+
+def kmq_probe_launch(stream=None, check=True) -> int:
+    """Enqueue the do-nothing kernel (the fixed cost of a call)."""
+    st = lib().kmq_probe_launch(_stream(stream))
+    if check:
+        _check(st, "kmq_probe_launch")
+    return st
+
+
+def kmq_probe_read_out_bytes() -> int:
+    return lib().kmq_probe_read_out_bytes()
+
+
+def kmq_probe_read(buf, nbytes, out, stream=None, check=True) -> int:
+    """Read `nbytes` of `buf` once with streaming loads (the read-only bandwidth ceiling)."""
+    st = lib().kmq_probe_read(_addr(buf), nbytes, _addr(out), _stream(stream))
+    if check:
+        _check(st, "kmq_probe_read")
     return st
