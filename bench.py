@@ -283,6 +283,148 @@ def machine_probes(torch, kmq, stream):
 EXTRA_CASES = [(n, N, K, b, M) for (n, N, K, _d, b, M) in WORKLOADS["large"]]
 
 
+# --------------------------------------------------------------------------
+# whole decode step: every backbone linear of a Llama-style model, one CUDA graph per token
+# --------------------------------------------------------------------------
+# Model shapes from the paper's table of architectures (appendix "Optimization Hyperparameters": width d, layers L,
+# heads, KV heads; head size 128; SwiGLU with multiplier 1.3, i.e. hidden = 1.3 * 8/3 * d rounded up to a multiple
+# of 1024, which reproduces the printed parameter counts).  name -> (d, L, q heads, kv heads)
+DECODE_MODELS = {"decode_4b": (3072, 24, 24, 8), "decode_12b": (4096, 48, 32, 8), "decode_31b": (6144, 60, 48, 8)}
+# the paper's tokens/s at batch 1 on one L40S (864 GB/s), its own block-scaled format and Triton kernels: context only
+PAPER_TOKENS_PER_S = {"decode_4b": {16: 88.8, 4.25: 190.1, 1.25: 245.6}, "decode_12b": {16: 30.0, 4.25: 79.3, 1.25: 120.0},
+                      "decode_31b": {4.25: 35.4, 1.25: 60.7}}
+
+
+def decode_layer_shapes(model):
+    d, L, heads, kv = DECODE_MODELS[model]
+    hidden = -(-int(1.3 * 8 * d / 3) // 1024) * 1024
+    qkv = (heads + 2 * kv) * 128
+    # (name, N out, K in, input: index of the call of the same layer whose output it reads, or -1 = the layer input)
+    return L, [("qkv", qkv, d, -1), ("o", d, d, 0), ("gate", hidden, d, 1), ("up", hidden, d, 1), ("down", d, hidden, 2)]
+
+
+def run_decode(args):
+    """All backbone linears of one decoding step (batch 1) as one CUDA graph: L layers x (QKV, O, gate, up, down),
+    every matrix with its own packed weights (random indices: timing does not depend on the values) and codebooks, the
+    calls chained through their activations wherever the shapes of the model chain them (attention, normalisation and
+    the activation function are not part of this library and are left out).  Reports tokens/s-equivalent = graph
+    replays per second and the effective bandwidth over the algorithmic bytes of all calls."""
+    import torch
+    from paper_2602_15563_b200 import build as kb
+    from paper_2602_15563_b200 import kmq, synth
+    from oracle import kmq_oracle as orc
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libkmq has no CPU path")
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    kb.build()
+    dev = torch.device("cuda")
+    peak_gbs, peak_kind = measured_peak()
+    L, shapes = decode_layer_shapes(args.workload)
+    d = DECODE_MODELS[args.workload][0]
+    results = []
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    stream = torch.cuda.Stream()
+    for bits in (1, 4):
+        g = torch.Generator(device=dev).manual_seed(bits)
+        calls, step_bytes, ws_bytes = [], 0, 16
+        x0 = (torch.randn(d, device=dev, generator=g)).to(torch.bfloat16).view(torch.int16)
+        for layer in range(L):
+            outs = []
+            for ci, (name, N, K, src) in enumerate(shapes):
+                layout = kmq.kmq_preferred_layout(N, K, bits, 1)
+                words = kmq.kmq_packed_bytes(N, K, bits, layout) // 4
+                if layer == 0:       # packed by kmq_pack from explicit indices: these calls are checked against the oracle
+                    idx = torch.randint(0, 1 << bits, (N, K), dtype=torch.uint8, device=dev, generator=g)
+                    packed = torch.empty(words, dtype=torch.int32, device=dev)
+                    kmq.kmq_pack(idx, N, K, bits, packed, layout=layout)
+                    rows = np.unique(np.concatenate([np.arange(16), np.arange(N - 16, N)]))
+                    check = (rows, idx[torch.from_numpy(rows).to(dev)].cpu().numpy())
+                    del idx
+                else:                # any bit pattern is a valid set of indices
+                    packed = torch.randint(-2**31, 2**31 - 1, (words,), dtype=torch.int32, device=dev, generator=g)
+                    check = None
+                cb = (torch.randn(N, 1 << bits, device=dev, generator=g) * 0.02).sort(dim=1).values
+                cb = cb.to(torch.bfloat16).view(torch.int16)
+                y = torch.zeros(N, dtype=torch.int16, device=dev)
+                x = (x0 if layer == 0 else calls[-1]["y"]) if src < 0 else outs[src]["y"]
+                ws_bytes = max(ws_bytes, kmq.kmq_workspace_bytes(N, K, bits, 1, layout))
+                c = {"name": name, "N": N, "K": K, "layout": layout, "packed": packed, "cb": cb, "x": x[:K], "y": y,
+                     "check": check, "variant": kmq.kmq_linear_variant(N, K, bits, 1, layout),
+                     "launches": kmq.kmq_linear_num_launches(N, K, bits, 1, layout)}
+                outs.append(c)
+                step_bytes += algorithmic_bytes(N, K, bits, 1)
+            calls += outs
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+
+        def issue():
+            for c in calls:
+                kmq.kmq_linear(c["packed"], c["cb"], c["x"], c["y"], c["N"], c["K"], bits, 1, ws, ws_bytes,
+                               layout=c["layout"])
+        with torch.cuda.stream(stream):
+            issue()
+            stream.synchronize()
+            # parity of the first layer's calls (the chain makes every input a previous output, also checked here)
+            worst = 0.0
+            for c in calls[:len(shapes)]:
+                rows, idx_rows = c["check"]
+                ref_packed = orc.pack_canonical(idx_rows, bits)
+                y_ref, s_abs = orc.linear_f64(ref_packed, c["cb"].cpu().numpy().view(np.uint16)[rows],
+                                              c["x"].cpu().numpy().view(np.uint16)[None, :], c["K"], bits)
+                got = c["y"].cpu().numpy().view(np.uint16)[None, rows]
+                worst = max(worst, orc.check_linear(got, y_ref, s_abs))
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                issue()
+            for _ in range(max(args.warmup, 3)):
+                graph.replay()
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            steps = max(1, min(args.steps, 50))
+            sampler.active = True
+            e0.record(stream)
+            for _ in range(steps):
+                graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+            sampler.active = False
+        ms = e0.elapsed_time(e1) / steps
+        variants = sorted({f"{c['name']}:{c['variant']}" for c in calls[:len(shapes)]})
+        results.append({"bits": bits, "ms_per_token": round(ms, 4), "tokens_per_s_equivalent": round(1e3 / ms, 1),
+                        "gbs": round(step_bytes / (ms * 1e-3) / 1e9, 1),
+                        "frac_of_measured_hbm": round(step_bytes / (ms * 1e-3) / 1e9 / peak_gbs, 4),
+                        "calls_per_token": len(calls), "launches_per_token": sum(c["launches"] for c in calls),
+                        "bytes_per_token": step_bytes, "variants": variants, "steps": steps,
+                        "parity_max_err_over_tol": round(worst, 4)})
+        del calls, outs, ws, graph
+        torch.cuda.empty_cache()
+    sampler.stop_flag = True
+    best = max(results, key=lambda r: r["gbs"])
+    line = {
+        "metric": "kmq_linear effective HBM bandwidth (algorithmic bytes / time), batch-1 k-means LUT GEMV",
+        "value": best["gbs"], "unit": "GB/s", "n_gpus": 1, "steps": best["steps"], "warmup": max(args.warmup, 3),
+        "ms_per_step": best["ms_per_token"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: every backbone linear of one decoding step at batch 1, "
+                               f"L = {L} layers x {[(n, N, K) for (n, N, K, _s) in shapes]}, one CUDA graph per token, "
+                               "distinct weights per matrix (far larger than L2), random indices",
+                   "multi_gpu": "replicas only"},
+        "per_bits": results,
+        "roofline": {"bound": "hbm", "kernel": "all kmq_linear calls of a token", "achieved": best["gbs"],
+                     "peak": peak_gbs, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": round(best["gbs"] / peak_gbs, 4), "traffic": None},
+        "gpu_launches": sum(r["launches_per_token"] * r["steps"] for r in results),
+        "clocks": sampler.summary(),
+        "parity": {"ok": all(r["parity_max_err_over_tol"] <= 1.0 for r in results)},
+        "paper_context": {"note": "paper's tokens/s for the whole model (attention, norms and bf16 embeddings included) "
+                                  "at batch 1 on one L40S (864 GB/s), by bits per weight; context only",
+                          "tokens_per_s": {str(k): v for k, v in PAPER_TOKENS_PER_S[args.workload].items()}},
+    }
+    print(json.dumps(line))
+
+
 def run_library(args):
     import torch
     from paper_2602_15563_b200 import build as kb
@@ -626,7 +768,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="kmq", choices=["kmq", "reference"])
-    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS) + sorted(DECODE_MODELS))
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--case", default="", help='subset of the workload, e.g. "bits=1,M=1" (keys: layer, N, K, bits, M)')
     ap.add_argument("--layout", default="auto", choices=["auto", "tuned", "table", "canonical"],
@@ -637,7 +779,11 @@ def main():
                     help="kernel timing only (no end-to-end leg, CPU baseline or parity check): for profiler runs")
     args = ap.parse_args()
     if args.impl == "reference":
+        if args.workload in DECODE_MODELS:
+            raise SystemExit("the reference arm times the oracle on the layer workloads (config*, tiny, large)")
         run_reference(args)
+    elif args.workload in DECODE_MODELS:
+        run_decode(args)
     else:
         run_library(args)
 
