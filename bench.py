@@ -425,6 +425,143 @@ def run_decode(args):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------
+# large batches: the fused kernel against "dequantise, then a standard bf16 GEMM"
+# --------------------------------------------------------------------------
+LARGE_BATCH_SHAPES = [("square8192", 8192, 8192, 2), ("gate_up", 16384, 3072, 2)]
+LARGE_BATCH_M = (16, 32, 64, 96, 128, 256, 512, 1024)
+
+
+def run_large_batch(args):
+    """Where the fused dequantise-multiply stops paying (paper, Section 3.3: the regimes below the theoretical
+    speed-up; appendix "Benchmarking": at large batch "dequantize in a separate kernel, before using a standard
+    high-precision GEMM").  Per shape and batch: kmq_linear; kmq_dequant_to_bf16 followed by a bf16 GEMM of the
+    vendor library (torch.matmul; a baseline leg, not a path of this library); that GEMM alone on resident bf16
+    weights (the 16-bit baseline).  The measured crossover is set beside the roofline model's P_w * nu / 16."""
+    import torch
+    from paper_2602_15563_b200 import build as kb
+    from paper_2602_15563_b200 import kmq
+    from oracle import kmq_oracle as orc
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libkmq has no CPU path")
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    kb.build()
+    dev = torch.device("cuda")
+    peak_gbs, peak_kind = measured_peak()
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            tflops = float(json.load(f)["bf16_tflops_sustained"])
+        tf_kind = "measured"
+    except Exception:
+        tflops, tf_kind = 1400.0, "fallback"
+    nu = tflops * 1e12 / (peak_gbs * 1e9)                    # the paper's nu = R_compute / R_transfer, flop per byte
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    stream = torch.cuda.Stream()
+    T = kmq.KMQ_LAYOUT_TUNED
+    rows_out, launches, worst = [], 0, 0.0
+    steps = max(1, min(args.steps, 20))
+    for (name, N, K, bits) in LARGE_BATCH_SHAPES:
+        g = torch.Generator(device=dev).manual_seed(N + K)
+        pool = max(4, -(-2 * L2_BYTES // (N * K * bits // 8)))
+        idx = torch.randint(0, 1 << bits, (N, K), dtype=torch.uint8, device=dev, generator=g)
+        packed = torch.empty((pool, kmq.kmq_packed_bytes(N, K, bits, T) // 4), dtype=torch.int32, device=dev)
+        kmq.kmq_pack(idx, N, K, bits, packed[0], layout=T)
+        packed[1:] = packed[0]
+        check_rows = np.unique(np.concatenate([np.arange(16), np.arange(N - 16, N)]))
+        ref_packed = orc.pack_canonical(idx[torch.from_numpy(check_rows).to(dev)].cpu().numpy(), bits)
+        del idx
+        cb = (torch.randn(N, 1 << bits, device=dev, generator=g) * 0.02).sort(dim=1).values.to(torch.bfloat16)
+        Wd = torch.empty((2, N, K), dtype=torch.bfloat16, device=dev)      # dequantised weights, two in rotation
+        kmq.kmq_dequant_to_bf16(packed[0], cb, Wd[0], N, K, bits, layout=T)
+        Wd[1] = Wd[0]
+        p_w = bits + 16.0 * (1 << bits) / K
+        for M in LARGE_BATCH_M:
+            x = torch.randn(M, K, device=dev, generator=g).to(torch.bfloat16)
+            y = torch.zeros(M, N, dtype=torch.bfloat16, device=dev)
+            y2 = torch.zeros(M, N, dtype=torch.bfloat16, device=dev)
+            ws_bytes = kmq.kmq_workspace_bytes(N, K, bits, M, T)
+            ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
+
+            def fused(i):
+                kmq.kmq_linear(packed[i % pool], cb, x, y, N, K, bits, M, ws, ws_bytes, layout=T)
+
+            def dequant_gemm(i):
+                kmq.kmq_dequant_to_bf16(packed[i % pool], cb, Wd[i % 2], N, K, bits, layout=T)
+                torch.matmul(x, Wd[i % 2].t(), out=y2)
+
+            def gemm_only(i):
+                torch.matmul(x, Wd[i % 2].t(), out=y2)
+            times = {}
+            with torch.cuda.stream(stream):
+                for leg, fn, reps in (("fused", fused, pool), ("dequant_gemm", dequant_gemm, 4), ("gemm_bf16", gemm_only, 4)):
+                    fn(0)
+                    stream.synchronize()
+                    gr = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(gr, stream=stream):
+                        for i in range(reps):
+                            fn(i)
+                    for _ in range(3):
+                        gr.replay()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    sampler.active = True
+                    e0.record(stream)
+                    for _ in range(steps):
+                        gr.replay()
+                    e1.record(stream)
+                    stream.synchronize()
+                    sampler.active = False
+                    times[leg] = e0.elapsed_time(e1) * 1e3 / (steps * reps)
+                    if leg == "fused":
+                        launches += steps * reps * kmq.kmq_linear_num_launches(N, K, bits, M, T)
+                # parity of the fused result (the last call used packed[(pool - 1) % pool] = the same weights)
+                y_ref, s_abs = orc.linear_f64(ref_packed, cb.view(torch.int16).cpu().numpy().view(np.uint16)[check_rows],
+                                              x.view(torch.int16).cpu().numpy().view(np.uint16), K, bits)
+                got = y[:, torch.from_numpy(check_rows).to(dev)].view(torch.int16).cpu().numpy().view(np.uint16)
+                worst = max(worst, orc.check_linear(got, y_ref, s_abs))
+            flops = 2.0 * M * N * K
+            rows_out.append({"layer": name, "N": N, "K": K, "bits": bits, "M": M,
+                             "variant": kmq.kmq_linear_variant(N, K, bits, M, T),
+                             "fused_us": round(times["fused"], 2), "dequant_gemm_us": round(times["dequant_gemm"], 2),
+                             "gemm_bf16_us": round(times["gemm_bf16"], 2),
+                             "fused_tflops": round(flops / times["fused"] / 1e6, 1),
+                             "fused_gbs": round(algorithmic_bytes(N, K, bits, M) / times["fused"] / 1e3, 1),
+                             "fused_faster_than_dequant_gemm": bool(times["fused"] < times["dequant_gemm"]),
+                             "fused_faster_than_bf16_gemm": bool(times["fused"] < times["gemm_bf16"]),
+                             "model_memory_bound_up_to_m": round(p_w * nu / 16.0, 1)})
+        del packed, Wd
+        torch.cuda.empty_cache()
+    sampler.stop_flag = True
+    cross = {}
+    for (name, N, K, bits) in LARGE_BATCH_SHAPES:
+        ms = [r["M"] for r in rows_out if r["layer"] == name and not r["fused_faster_than_dequant_gemm"]]
+        cross[name] = min(ms) if ms else None
+    best = max(rows_out, key=lambda r: r["fused_tflops"])
+    line = {
+        "metric": "kmq_linear effective HBM bandwidth (algorithmic bytes / time), batch-1 k-means LUT GEMV",
+        "value": best["fused_gbs"], "unit": "GB/s", "n_gpus": 1, "steps": steps, "warmup": 3,
+        "ms_per_step": round(best["fused_us"] * 1e-3, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "large_batch: fused kmq_linear against kmq_dequant_to_bf16 + bf16 GEMM and against the "
+                               "bf16 GEMM alone, batches " + str(list(LARGE_BATCH_M)) + " on "
+                               + str([(n, N, K, b) for (n, N, K, b) in LARGE_BATCH_SHAPES]) + ", random indices",
+                   "l2": "packed weights from a pool larger than 2 x L2; dequantised weights: two buffers in rotation",
+                   "multi_gpu": "replicas only"},
+        "per_case": rows_out,
+        "first_batch_where_dequant_plus_gemm_wins": cross,
+        "roofline_model": {"nu_flop_per_byte": round(nu, 1), "tensor_tflops": tflops, "tensor_kind": f"of {tf_kind}",
+                           "hbm_gbs": peak_gbs, "rule": "memory bound while m < P_w * nu / 16 (paper, theoretical model)"},
+        "roofline": {"bound": "tensor", "kernel": f"kmq_linear[{best['variant']}] M={best['M']} {best['N']}x{best['K']}",
+                     "achieved": best["fused_tflops"], "peak": tflops, "peak_kind": f"of {tf_kind} (sustained bf16)",
+                     "unit": "TFLOP/s", "frac": round(best["fused_tflops"] / tflops, 4), "traffic": None},
+        "gpu_launches": launches, "clocks": sampler.summary(),
+        "parity": {"max_err_over_tol": round(worst, 4), "ok": bool(worst <= 1.0)},
+    }
+    print(json.dumps(line))
+
+
 def run_library(args):
     import torch
     from paper_2602_15563_b200 import build as kb
@@ -768,7 +905,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="kmq", choices=["kmq", "reference"])
-    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS) + sorted(DECODE_MODELS))
+    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS) + sorted(DECODE_MODELS) + ["large_batch"])
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--case", default="", help='subset of the workload, e.g. "bits=1,M=1" (keys: layer, N, K, bits, M)')
     ap.add_argument("--layout", default="auto", choices=["auto", "tuned", "table", "canonical"],
@@ -779,11 +916,13 @@ def main():
                     help="kernel timing only (no end-to-end leg, CPU baseline or parity check): for profiler runs")
     args = ap.parse_args()
     if args.impl == "reference":
-        if args.workload in DECODE_MODELS:
+        if args.workload in DECODE_MODELS or args.workload == "large_batch":
             raise SystemExit("the reference arm times the oracle on the layer workloads (config*, tiny, large)")
         run_reference(args)
     elif args.workload in DECODE_MODELS:
         run_decode(args)
+    elif args.workload == "large_batch":
+        run_large_batch(args)
     else:
         run_library(args)
 
