@@ -64,7 +64,7 @@ __device__ __forceinline__ int piece_offset(int w) {
 template <int BITS, int MMAX>
 __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed, const uint16_t* __restrict__ cb,
                                              const uint16_t* __restrict__ x, int64_t N, int64_t K, int M,
-                                             int64_t tile_id, int sa, int sb, float& v) {
+                                             int64_t tile_id, int sa, int sb, bool wait_for_x, float& v) {
   using G = TGeo<BITS>;
   using SM = TSmem<BITS, MMAX>;
   constexpr int Q = G::kMmaPerWord;
@@ -120,7 +120,6 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
     if (s < sb) {
       qa[d] = ldg_stream_u4(tile + (int64_t)s * 64);
       qb[d] = ldg_stream_u4(tile + (int64_t)s * 64 + 32);
-      if constexpr (kPrefetchX) load_x(s, qx[kPrefetchX ? d : 0]);
     }
   }
 
@@ -156,6 +155,26 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
     __syncthreads();
   }
   const uint32_t lane4 = lane * 4;
+
+  // Programmatic dependent launch: up to here only the packed indices and the codebooks were read, which are
+  // constants of the layer; the activations may come from the previous kernel on the stream, so they are read
+  // only once that kernel is known to have completed.  A CTA that became resident early has its first weights
+  // under way (and, for b = 4, its tables built) by then.
+  if (wait_for_x) {
+    // a hint only (it binds no value): the first few CTAs pull the activations towards L2 while waiting
+    if (blockIdx.x < 4) {
+      for (int64_t o = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 64; o < (int64_t)M * K; o += 4 * kThreads * 64)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(x + o));
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+  }
+  if constexpr (kPrefetchX) {
+#pragma unroll
+    for (int d = 0; d < STAGES; ++d) {
+      const int s = sa + warp + d * kWarps;
+      if (s < sb) load_x(s, qx[d]);
+    }
+  }
 
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
 
@@ -252,14 +271,13 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) linear_tiled_kernel(c
                                                                     const uint16_t* __restrict__ x,
                                                                     uint16_t* __restrict__ y, int64_t N, int64_t K,
                                                                     int M) {
-  // Programmatic dependent launch: nothing is read before the previous kernel on the stream has completed (same
-  // ordering as a plain launch), but this grid could be set up while that kernel drained, and the next kernel may be
-  // set up while this one sums and stores.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int steps = (int)((K / (4 * TGeo<BITS>::kWordK) + 3) >> 2);
   const int64_t row0 = (int64_t)blockIdx.x * kRows;
   float v;
-  tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, blockIdx.x, 0, steps, v);
+  tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, blockIdx.x, 0, steps, true, v);
+  // Programmatic dependent launch: from here on the next kernel on the stream may become resident; it reads nothing
+  // but constants of its layer until this kernel has completed (see tile_segment), so its first weights are under
+  // way while this one stores and drains.
   asm volatile("griddepcontrol.launch_dependents;");
   store_output(v, y, N, M, row0);
 }
@@ -286,7 +304,7 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) linear_split_kernel(c
     const int64_t base = tile * steps;
     const int sa = (int)(u0 > base ? u0 - base : 0), sb = (int)(u1 - base < steps ? u1 - base : steps);
     float v;
-    tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, tile, sa, sb, v);
+    tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, tile, sa, sb, false, v);
     if (sa == 0 && sb == steps) {
       store_output(v, y, N, M, tile * kRows);
     } else if (threadIdx.x < kRows * 8) {
