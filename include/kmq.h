@@ -122,8 +122,9 @@ size_t kmq_workspace_bytes(int64_t N, int64_t K, int bits, int64_t M, int layout
 
 /* Number of kernels one kmq_linear call launches for this shape (one per pass
  * of batch rows; 2 for the balanced split with its fix-up kernel), and a short
- * static name of the kernel variant the dispatcher picks: "tiled_*", "split_*",
- * "multi_*", "tcgen05_*" (tuned layout), "staged_*" (canonical layout),
+ * static name of the kernel variant the dispatcher picks: "tiled_*",
+ * "split_*", "multi_*", "tcgen05_*" (tuned layout), "table_*" (table layout,
+ * bits = 1, 2), "staged_*" (canonical layout),
  * "generic_warp_per_row", or "invalid". */
 int kmq_linear_num_launches(int64_t N, int64_t K, int bits, int64_t M, int layout);
 const char* kmq_linear_variant(int64_t N, int64_t K, int bits, int64_t M, int layout);
