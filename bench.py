@@ -562,6 +562,114 @@ def run_large_batch(args):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------
+# the paper's own block format (shared codebook + bf16 scale per block of 64)
+# --------------------------------------------------------------------------
+BLOCK_CASES = [(4096, 4096, b, 1) for b in (1, 2, 4, 8)] + [(8192, 8192, b, 1) for b in (1, 4)]
+
+
+def block_bytes(N, K, bits, M):
+    """Algorithmic bytes of one kmq_block_linear call: P_w = bits + 16/64 bits per weight (indices + scales), the
+    codebook, activations in, outputs out."""
+    return N * K * bits // 8 + N * (K // 64) * 2 + (1 << bits) * 2 + M * K * 2 + M * N * 2
+
+
+def run_block(args):
+    """kmq_block_linear (deferred scaling) at batch 1 on the paper's micro-benchmark shape (8192 x 8192) and on
+    4096 x 4096, random indices and scales (timing does not depend on the values), pool of weight sets larger than
+    2 x L2, one CUDA graph per case."""
+    import torch
+    from paper_2602_15563_b200 import build as kb
+    from paper_2602_15563_b200 import kmq
+    from oracle import kmq_block_oracle as blk
+    from oracle import kmq_oracle as orc
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libkmq has no CPU path")
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    kb.build()
+    dev = torch.device("cuda")
+    peak_gbs, peak_kind = measured_peak()
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    stream = torch.cuda.Stream()
+    steps = max(1, min(args.steps, 50))
+    rows_out, launches, worst = [], 0, 0.0
+    for (N, K, bits, M) in BLOCK_CASES:
+        g = torch.Generator(device=dev).manual_seed(N + 7 * bits)
+        nbytes = block_bytes(N, K, bits, M)
+        pool = max(4, -(-2 * L2_BYTES // nbytes))
+        idx = torch.randint(0, 1 << bits, (N, K), dtype=torch.uint8, device=dev, generator=g)
+        wq = torch.empty((pool, N * K * bits // 8), dtype=torch.uint8, device=dev)
+        kmq.kmq_block_pack(idx, N, K, bits, wq[0])
+        wq[1:] = wq[0]
+        rows = np.unique(np.concatenate([np.arange(16), np.arange(N - 16, N)]))
+        ref_wq = blk.pack_bytes(idx[torch.from_numpy(rows).to(dev)].cpu().numpy(), bits)
+        del idx
+        scales = (torch.rand(N, K // 64, device=dev, generator=g) * 0.05 + 0.01).to(torch.bfloat16)
+        cb = torch.linspace(-1, 1, 1 << bits, device=dev).to(torch.bfloat16)
+        x = torch.randn(pool, M, K, device=dev, generator=g).to(torch.bfloat16)
+        y = torch.zeros(pool, M, N, dtype=torch.bfloat16, device=dev)
+
+        def call(i):
+            kmq.kmq_block_linear(wq[i], scales, cb, x[i], y[i], N, K, bits, M, scale_order=kmq.KMQ_SCALE_DEFERRED)
+        with torch.cuda.stream(stream):
+            call(0)
+            stream.synchronize()
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr, stream=stream):
+                for i in range(pool):
+                    call(i)
+            for _ in range(max(args.warmup, 3)):
+                gr.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            sampler.active = True
+            e0.record(stream)
+            for _ in range(steps):
+                gr.replay()
+            e1.record(stream)
+            stream.synchronize()
+            sampler.active = False
+        us = e0.elapsed_time(e1) * 1e3 / (steps * pool)
+        launches += steps * pool
+        for i in (0, pool - 1):
+            y_ref, s_abs = blk.block_linear_f64(ref_wq, scales.view(torch.int16).cpu().numpy().view(np.uint16)[rows],
+                                                cb.view(torch.int16).cpu().numpy().view(np.uint16),
+                                                x[i].view(torch.int16).cpu().numpy().view(np.uint16), K, bits)
+            got = y[i][:, torch.from_numpy(rows).to(dev)].view(torch.int16).cpu().numpy().view(np.uint16)
+            worst = max(worst, orc.check_linear(got, y_ref, s_abs))
+        gbs = nbytes / us / 1e3
+        rows_out.append({"N": N, "K": K, "bits": bits, "P_w": bits + 0.25, "M": M, "pool": pool, "us_per_call": round(us, 3),
+                         "gbs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peak_gbs, 4), "bytes_per_call": nbytes,
+                         "ideal_us_at_measured_hbm": round(nbytes / (peak_gbs * 1e3), 3)})
+        del wq, x, y
+        torch.cuda.empty_cache()
+    sampler.stop_flag = True
+    tot_b = sum(r["bytes_per_call"] * r["pool"] for r in rows_out)
+    tot_us = sum(r["us_per_call"] * r["pool"] for r in rows_out)
+    dom = max(rows_out, key=lambda r: r["us_per_call"] * r["pool"])
+    line = {
+        "metric": "kmq_linear effective HBM bandwidth (algorithmic bytes / time), batch-1 k-means LUT GEMV",
+        "value": round(tot_b / tot_us / 1e3, 2), "unit": "GB/s", "n_gpus": 1, "steps": steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(tot_us * 1e-3, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "block: the paper's k-means block format (shared codebook, bf16 scale per block of 64, "
+                               "P_w = b + 0.25), kmq_block_linear with deferred scaling at batch 1 on "
+                               + str([(N, K, b) for (N, K, b, _m) in BLOCK_CASES]) + ", random indices and scales",
+                   "l2": "inputs larger than L2: every call of a step uses its own weight set, pool >= 2 x 126 MB",
+                   "multi_gpu": "replicas only"},
+        "per_case": rows_out,
+        "roofline": {"bound": "hbm", "kernel": f"kmq_block_linear b={dom['bits']} {dom['N']}x{dom['K']}",
+                     "achieved": dom["gbs"], "peak": peak_gbs, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": dom["frac_of_measured_hbm"], "traffic": None},
+        "gpu_launches": launches, "clocks": sampler.summary(),
+        "parity": {"max_err_over_tol": round(worst, 4), "ok": bool(worst <= 1.0)},
+        "paper_context": PAPER_CONTEXT,
+    }
+    print(json.dumps(line))
+
+
 def run_library(args):
     import torch
     from paper_2602_15563_b200 import build as kb
@@ -905,7 +1013,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="kmq", choices=["kmq", "reference"])
-    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS) + sorted(DECODE_MODELS) + ["large_batch"])
+    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS) + sorted(DECODE_MODELS) + ["large_batch", "block"])
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--case", default="", help='subset of the workload, e.g. "bits=1,M=1" (keys: layer, N, K, bits, M)')
     ap.add_argument("--layout", default="auto", choices=["auto", "tuned", "table", "canonical"],
@@ -916,13 +1024,15 @@ def main():
                     help="kernel timing only (no end-to-end leg, CPU baseline or parity check): for profiler runs")
     args = ap.parse_args()
     if args.impl == "reference":
-        if args.workload in DECODE_MODELS or args.workload == "large_batch":
+        if args.workload in DECODE_MODELS or args.workload in ("large_batch", "block"):
             raise SystemExit("the reference arm times the oracle on the layer workloads (config*, tiny, large)")
         run_reference(args)
     elif args.workload in DECODE_MODELS:
         run_decode(args)
     elif args.workload == "large_batch":
         run_large_batch(args)
+    elif args.workload == "block":
+        run_block(args)
     else:
         run_library(args)
 

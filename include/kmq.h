@@ -265,6 +265,44 @@ kmq_status kmq_dequant_to_bf16(const uint32_t* packed, const uint16_t* codebooks
                                int64_t N, int64_t K, int bits, int layout, void* stream);
 
 /*
+ * The paper's own k-means block format (Section 2.1 "Block formats", Eq.
+ * "fractional bit width"; Section 2.2 "Nonlinear k-means quantization";
+ * Appendix "Benchmarking", "Kernel implementations"): one codebook of 2^bits
+ * centroids per weight tensor (bits = 1, 2, 4 or 8) and one bf16 scale per
+ * block of 64 consecutive inputs of an output row,
+ *     W^[n, k] = scale[n, k/64] * c[idx[n, k]],     P_w = bits + 16/64 bits per weight.
+ *   wq       DEVICE uint8 [N, K*bits/8] row-major: the indices packed along the
+ *            input dimension, 8/bits per byte, field i of a byte at bits
+ *            [i*bits, (i+1)*bits) (the paper leaves the order inside a byte
+ *            open; LSB first is the reading taken here).
+ *   scales   DEVICE bf16 [N, K/64] row-major.
+ *   codebook DEVICE bf16 [2^bits].
+ * K must be a multiple of 64; all pointers 16-byte aligned.
+ *
+ * kmq_block_pack -- idx DEVICE uint8 [N, K] (low `bits` bits kept) -> wq.
+ * kmq_block_linear -- y[m,n] = sum_k x[m,k] * W^[n,k], fp32 accumulation,
+ *   bf16 result.  scale_order picks between the paper's two listings:
+ *   KMQ_SCALE_DIRECT multiplies every centroid by its block's scale before the
+ *   multiply-accumulate; KMQ_SCALE_DEFERRED ("deferred scaling") accumulates
+ *   the 64 unscaled products of a block and scales their sum.  Both are the
+ *   same sum up to fp32 rounding and both meet the tolerance stated for
+ *   kmq_linear.  x DEVICE bf16 [M,K], y DEVICE bf16 [M,N]; no workspace.
+ * kmq_block_dequant_to_bf16 -- W DEVICE bf16 [N,K] = bf16(scale * centroid):
+ *   the exact product rounded once, to nearest even (the separate dequantise
+ *   step ahead of a standard GEMM, Appendix "Benchmarking", "Model benchmarks").
+ * Errors: KMQ_ERR_NULL, KMQ_ERR_BITS, KMQ_ERR_SHAPE, KMQ_ERR_ALIGN,
+ * KMQ_ERR_LAYOUT (unknown scale_order), KMQ_ERR_CUDA.
+ */
+#define KMQ_SCALE_DIRECT 0
+#define KMQ_SCALE_DEFERRED 1
+size_t kmq_block_packed_bytes(int64_t N, int64_t K, int bits);
+kmq_status kmq_block_pack(const uint8_t* idx, int64_t N, int64_t K, int bits, uint8_t* wq, void* stream);
+kmq_status kmq_block_linear(const uint8_t* wq, const uint16_t* scales, const uint16_t* codebook, const uint16_t* x,
+                            uint16_t* y, int64_t N, int64_t K, int bits, int64_t M, int scale_order, void* stream);
+kmq_status kmq_block_dequant_to_bf16(const uint8_t* wq, const uint16_t* scales, const uint16_t* codebook, uint16_t* W,
+                                     int64_t N, int64_t K, int bits, void* stream);
+
+/*
  * Measurement helpers (conveniences of this library; the paper has no
  * counterpart).  They put the layer's timings into proportion on the GPU at
  * hand:

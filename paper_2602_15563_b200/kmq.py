@@ -21,6 +21,7 @@ KMQ_ERR_SCRATCH_LIMIT = 8
 KMQ_LAYOUT_CANONICAL = 0
 KMQ_LAYOUT_TUNED = 1
 KMQ_LAYOUT_TABLE = 2
+KMQ_SCALE_DIRECT, KMQ_SCALE_DEFERRED = 0, 1
 KMQ_DEVICE_ERROR_WAIT_TIMEOUT = 1
 KMQ_DEVICE_ERROR_SMEM_WINDOW = 2
 
@@ -47,6 +48,10 @@ SIGNATURES = {
     "kmq_linear_tcgen05": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _ptr]),
     "kmq_device_error_flags": (_int, [_ptr]),
     "kmq_dequant_to_bf16": (_int, [_ptr, _ptr, _ptr, _i64, _i64, _int, _int, _ptr]),
+    "kmq_block_packed_bytes": (_sz, [_i64, _i64, _int]),
+    "kmq_block_pack": (_int, [_ptr, _i64, _i64, _int, _ptr, _ptr]),
+    "kmq_block_linear": (_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr]),
+    "kmq_block_dequant_to_bf16": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _ptr]),
     "kmq_probe_launch": (_int, [_ptr]),
     "kmq_probe_read_out_bytes": (_sz, []),
     "kmq_probe_read": (_int, [_ptr, _sz, _ptr, _ptr]),
@@ -226,4 +231,33 @@ def kmq_probe_read(buf, nbytes, out, stream=None, check=True) -> int:
     st = lib().kmq_probe_read(_addr(buf), nbytes, _addr(out), _stream(stream))
     if check:
         _check(st, "kmq_probe_read")
+    return st
+
+
+def kmq_block_packed_bytes(N, K, bits) -> int:
+    return lib().kmq_block_packed_bytes(N, K, bits)
+
+
+def kmq_block_pack(idx, N, K, bits, wq, stream=None, check=True) -> int:
+    st = lib().kmq_block_pack(_addr(idx), N, K, bits, _addr(wq), _stream(stream))
+    if check:
+        _check(st, "kmq_block_pack")
+    return st
+
+
+def kmq_block_linear(wq, scales, codebook, x, y, N, K, bits, M, scale_order=KMQ_SCALE_DEFERRED, stream=None,
+                     check=True) -> int:
+    """The paper's block format (shared codebook, bf16 scale per block of 64): y = x * W^T."""
+    st = lib().kmq_block_linear(_addr(wq), _addr(scales), _addr(codebook), _addr(x), _addr(y), N, K, bits, M,
+                                scale_order, _stream(stream))
+    if check:
+        _check(st, "kmq_block_linear")
+    return st
+
+
+def kmq_block_dequant_to_bf16(wq, scales, codebook, W, N, K, bits, stream=None, check=True) -> int:
+    st = lib().kmq_block_dequant_to_bf16(_addr(wq), _addr(scales), _addr(codebook), _addr(W), N, K, bits,
+                                         _stream(stream))
+    if check:
+        _check(st, "kmq_block_dequant_to_bf16")
     return st

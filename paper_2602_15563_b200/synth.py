@@ -179,6 +179,38 @@ def make_layer(N: int, K: int, bits: int, M: int, dist: str = "normal",
 
 # (name, N, K, distribution) for the benchmark configurations; bits and batch
 # sizes are chosen by the caller.
+def make_block_layer(N: int, K: int, bits: int, M: int, dist: str = "normal", config_id: int = 0,
+                     fit_samples: int = 1 << 20) -> dict:
+    """Synthetic layer in the paper's k-means block format (Section 2.2): one bf16 scale per block of 64 inputs of a
+    row (absmax of the block; a block of zeros gets scale 1), the weights divided by their stored scale lie in
+    [-1, 1], one codebook of 2^bits centroids per tensor from 1-D Lloyd (same rules as lloyd_rows: quantile start,
+    20 iterations) on an evenly strided sample of at most `fit_samples` normalised weights, indices = nearest stored
+    centroid (ties and duplicates to the lowest index).  Input generation only: nothing here is on the timed path.
+    Returns idx uint8 [N, K], scales bf16 bits [N, K/64], codebook bf16 bits [2^bits], x bf16 bits [M, K], W fp32."""
+    if K % 64:
+        raise ValueError("K must be a multiple of 64")
+    W = draw_weights(dist, N, K, rng_for(config_id, TENSOR_W))
+    blocks = W.reshape(N, K // 64, 64).astype(np.float64)
+    absmax = np.abs(blocks).max(axis=2)
+    scales = f32_to_bf16_bits(np.where(absmax > 0, absmax, 1.0).astype(np.float32))
+    s64 = bf16_bits_to_f32(scales).astype(np.float64)
+    # bf16 rounding may bring the stored scale just below the block's absmax: clip the ratio into [-1, 1]
+    norm = np.clip(blocks / s64[:, :, None], -1.0, 1.0).reshape(N, K)
+    flat = norm.reshape(1, -1)
+    stride = max(1, flat.shape[1] // fit_samples)
+    cent = lloyd_rows(flat[:, ::stride], bits)                     # [1, 2^bits], sorted
+    codebook = f32_to_bf16_bits(cent.astype(np.float32))[0]
+    cb = bf16_bits_to_f32(codebook).astype(np.float64)
+    mids = 0.5 * (cb[:-1] + cb[1:])
+    first = np.arange(cb.size)
+    for i in range(1, cb.size):
+        if cb[i] == cb[i - 1]:
+            first[i] = first[i - 1]
+    idx = first[np.searchsorted(mids, norm, side="left")].astype(np.uint8)   # a weight on a midpoint stays below
+    x = draw_activations(M, K, rng_for(config_id, TENSOR_X))
+    return {"idx": idx, "scales": scales, "codebook": codebook, "x": x, "W": W}
+
+
 CONFIG_LAYERS = {
     1: [("tiny", 256, 256, "normal")],
     2: [("square4096", 4096, 4096, "normal")],

@@ -105,3 +105,19 @@ def test_distributions_and_determinism():
     assert a["idx"].max() < 4 and a["x"].shape == (3, 64) and a["codebooks"].shape == (32, 4)
     c = synth.make_layer(32, 64, 2, 3, "student_t", config_id=4)
     assert not np.array_equal(a["x"], c["x"])
+
+
+@pytest.mark.parametrize("bits", (1, 2, 4, 8))
+def test_block_layer_generator(bits):
+    """make_block_layer: scales are the stored absmax of each block, the codebook is sorted and inside [-1, 1], and
+    every index is the nearest stored centroid of the normalised weight (brute force, lowest index on ties)."""
+    L = synth.make_block_layer(24, 256, bits, 1, "normal", config_id=3)
+    W = L["W"].astype(np.float64).reshape(24, 4, 64)
+    s = synth.bf16_bits_to_f32(L["scales"]).astype(np.float64)
+    assert np.array_equal(L["scales"], synth.f32_to_bf16_bits(np.abs(L["W"]).reshape(24, 4, 64).max(axis=2)))
+    cb = synth.bf16_bits_to_f32(L["codebook"]).astype(np.float64)
+    assert cb.size == 1 << bits and np.all(np.diff(cb) >= 0) and cb.min() >= -1.0 and cb.max() <= 1.0
+    norm = np.clip(W / s[:, :, None], -1.0, 1.0).reshape(24, 256)
+    brute = np.abs(norm[:, :, None] - cb[None, None, :]).argmin(axis=2)        # argmin takes the first minimum
+    assert np.array_equal(L["idx"], brute)
+    assert L["idx"].max() < (1 << bits)
