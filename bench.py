@@ -676,6 +676,141 @@ def run_block(args):
     print(json.dumps(line))
 
 
+# (format, N, K, bits): "rows" = a codebook per row (kmq_quantize_rows), "block" = the paper's block format
+QUANTIZE_CASES = [("rows", 4096, 4096, 1), ("rows", 4096, 4096, 2), ("rows", 4096, 4096, 4), ("rows", 8192, 8192, 2),
+                  ("rows", 8192, 28672, 1), ("rows", 8192, 28672, 4), ("block", 4096, 4096, 4), ("block", 8192, 8192, 1)]
+QUANTIZE_SAMPLES = 32768
+
+
+def run_quantize(args):
+    """The quantiser side on the GPU: float32 weights -> codebooks (+ block scales) -> packed indices.  Seeded N(0,
+    0.02) weights drawn on the device; every timed call reads its own copy of the weights out of a pool larger than
+    L2.  The fit and the assignment are also timed on their own; sampled rows are checked against the oracle."""
+    import torch
+    from paper_2602_15563_b200 import build as kb
+    from paper_2602_15563_b200 import kmq
+    from oracle import kmq_block_oracle as blk
+    from oracle import kmq_quant_oracle as qorc
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libkmq has no CPU path")
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    kb.build()
+    dev = torch.device("cuda")
+    peak_gbs, peak_kind = measured_peak()
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    sampler.start()
+    stream = torch.cuda.Stream()
+    steps = max(1, min(args.steps, 10))
+    rows_out, launches, parity_ok = [], 0, True
+    cpu_rows_per_s = {}
+
+    def timed(fn, pool):
+        with torch.cuda.stream(stream):
+            for i in range(min(pool, max(args.warmup, 3))):
+                fn(i % pool)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for it in range(steps):
+                fn(it % pool)
+            e1.record(stream)
+            stream.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    for (fmt, N, K, bits) in QUANTIZE_CASES:
+        g = torch.Generator(device=dev).manual_seed(N + K + bits)
+        pool = max(2, -(-(L2_BYTES + L2_BYTES // 2) // (N * K * 4)))
+        W = torch.randn((pool, N, K), generator=g, device=dev, dtype=torch.float32) * 0.02
+        Q = 1 << bits
+        rows = np.unique(np.concatenate([[0, 15, 16, N - 1], np.random.default_rng(N).integers(0, N, 4)]))
+        sampler.active = True
+        if fmt == "rows":
+            layout = kmq.kmq_preferred_layout(N, K, bits, 1)
+            cb = torch.empty((N, Q), dtype=torch.int16, device=dev)
+            packed = torch.empty(kmq.kmq_packed_bytes(N, K, bits, layout) // 4, dtype=torch.int32, device=dev)
+            out_bytes = packed.numel() * 4 + cb.numel() * 2
+            ms_all = timed(lambda i: kmq.kmq_quantize_rows(W[i], N, K, bits, 20, layout, cb, packed, stream=stream), pool)
+            ms_fit = timed(lambda i: kmq.kmq_kmeans_rows(W[i], N, K, bits, 20, cb, stream=stream), pool)
+            ms_assign = timed(lambda i: kmq.kmq_assign_pack(W[i], cb, N, K, bits, layout, packed, stream=stream), pool)
+            launches += steps * 4
+            kmq.kmq_quantize_rows(W[0], N, K, bits, 20, layout, cb, packed, stream=stream)
+            idx = torch.empty((N, K), dtype=torch.uint8, device=dev)
+            kmq.kmq_unpack(packed, N, K, bits, idx, layout=layout, stream=stream)
+            stream.synchronize()
+            sel = torch.from_numpy(rows).to(dev)
+            w_rows = W[0][sel].cpu().numpy()
+            t0 = time.perf_counter()
+            want_cb = qorc.centroids_to_bf16(qorc.lloyd_rows(w_rows, bits))
+            want_idx = qorc.nearest_centroid(w_rows, want_cb)
+            cpu_rows_per_s[(N, K, bits)] = len(rows) / (time.perf_counter() - t0)
+            ok = (np.array_equal(cb[sel].cpu().numpy().view(np.uint16), want_cb)
+                  and np.array_equal(idx[sel].cpu().numpy(), want_idx))
+            del idx, packed
+        else:
+            scales = torch.empty(N * K // 64, dtype=torch.int16, device=dev)
+            cb = torch.empty(max(8, Q), dtype=torch.int16, device=dev)
+            wq = torch.empty(kmq.kmq_block_packed_bytes(N, K, bits), dtype=torch.uint8, device=dev)
+            ws = torch.empty(QUANTIZE_SAMPLES, dtype=torch.float32, device=dev)
+            out_bytes = wq.numel() + scales.numel() * 2 + Q * 2
+            lam = kmq.KMQ_LAMBDA_ABSMAX
+            ms_all = timed(lambda i: kmq.kmq_block_quantize(W[i], N, K, bits, lam, 20, QUANTIZE_SAMPLES, scales, cb, wq,
+                                                            ws, stream=stream), pool)
+            ms_fit = timed(lambda i: kmq.kmq_kmeans_rows(ws, 1, QUANTIZE_SAMPLES, bits, 20, cb, stream=stream), pool)
+            ms_assign = timed(lambda i: kmq.kmq_block_assign_pack(W[i], scales, cb, N, K, bits, wq, stream=stream), pool)
+            launches += steps * 6
+            kmq.kmq_block_quantize(W[0], N, K, bits, lam, 20, QUANTIZE_SAMPLES, scales, cb, wq, ws, stream=stream)
+            stream.synchronize()
+            w_rows = W[0][:256].cpu().numpy()
+            s_all = scales.cpu().numpy().view(np.uint16).reshape(N, K // 64)
+            cbn = cb.cpu().numpy().view(np.uint16)[:Q]
+            ok = (np.array_equal(s_all[:256], qorc.block_scales(w_rows, qorc.ABSMAX))
+                  and np.array_equal(wq.view(N, -1)[:256].cpu().numpy(),
+                                     blk.pack_bytes(qorc.block_assign(w_rows, s_all[:256], cbn), bits)))
+            del wq, scales
+        sampler.active = False
+        parity_ok = parity_ok and bool(ok)
+        nbytes = N * K * 4 + out_bytes
+        rows_out.append({"format": fmt, "N": N, "K": K, "bits": bits, "pool": pool, "ms_per_call": round(ms_all, 4),
+                         "ms_fit": round(ms_fit, 4), "ms_assign_pack": round(ms_assign, 4),
+                         "gbs": round(nbytes / ms_all / 1e6, 1), "frac_of_measured_hbm": round(nbytes / ms_all / 1e6 / peak_gbs, 4),
+                         "assign_pack_gbs": round(nbytes / ms_assign / 1e6, 1),
+                         "mweights_per_s": round(N * K / ms_all / 1e3, 1), "bytes_per_call": nbytes,
+                         "ideal_ms_at_measured_hbm": round(nbytes / (peak_gbs * 1e6), 4), "parity_ok": bool(ok)})
+        del W
+        torch.cuda.empty_cache()
+    sampler.stop_flag = True
+    tot_b = sum(r["bytes_per_call"] for r in rows_out)
+    tot_ms = sum(r["ms_per_call"] for r in rows_out)
+    dom = max(rows_out, key=lambda r: r["ms_per_call"])
+    key = (dom["N"], dom["K"], dom["bits"])
+    cpu = None
+    if key in cpu_rows_per_s:
+        cpu = {"value": round(cpu_rows_per_s[key] * dom["K"] / 1e6, 3), "unit": "Mweights/s", "cores": _cpu_threads(),
+               "kind": "oracle", "sample": f"lloyd_rows + nearest_centroid on 8 rows of the {dom['N']}x{dom['K']} b={dom['bits']} case"}
+    line = {
+        "metric": "quantiser throughput: float32 weights read + packed indices, codebooks and scales written, per second",
+        "value": round(tot_b / tot_ms / 1e6, 2), "unit": "GB/s", "n_gpus": 1, "steps": steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(tot_ms, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "quantize: per-row 1-D Lloyd fit (quantile start, 20 iterations) + nearest-centroid "
+                               "assignment + packing (kmq_quantize_rows), and the block format's scales + sampled "
+                               "shared-codebook fit + assignment (kmq_block_quantize, absmax, 32768 samples), on "
+                               + str([(f, N, K, b) for (f, N, K, b) in QUANTIZE_CASES]) + ", N(0, 0.02) float32 weights",
+                   "l2": "inputs larger than L2: consecutive calls read different copies of the weights, pool >= 1.5 x 126 MB",
+                   "multi_gpu": "replicas only"},
+        "per_case": rows_out,
+        "roofline": {"bound": "alu", "kernel": f"lloyd_rows_kernel {dom['N']}x{dom['K']} b={dom['bits']}",
+                     "note": "the fit is bound by the shared-memory sorting network, not by HBM; the fraction below is "
+                             "algorithmic bytes / time against the HBM peak for orientation",
+                     "achieved": dom["gbs"], "peak": peak_gbs, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": dom["frac_of_measured_hbm"], "traffic": None},
+        "gpu_launches": launches, "clocks": sampler.summary(), "cpu_baseline": cpu,
+        "parity": {"ok": parity_ok},
+    }
+    print(json.dumps(line))
+
+
 def run_library(args):
     import torch
     from paper_2602_15563_b200 import build as kb
@@ -1019,7 +1154,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="kmq", choices=["kmq", "reference"])
-    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS) + sorted(DECODE_MODELS) + ["large_batch", "block"])
+    ap.add_argument("--workload", default="config2", choices=sorted(WORKLOADS) + sorted(DECODE_MODELS) + ["large_batch", "block", "quantize"])
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--case", default="", help='subset of the workload, e.g. "bits=1,M=1" (keys: layer, N, K, bits, M)')
     ap.add_argument("--layout", default="auto", choices=["auto", "tuned", "table", "canonical"],
@@ -1030,7 +1165,7 @@ def main():
                     help="kernel timing only (no end-to-end leg, CPU baseline or parity check): for profiler runs")
     args = ap.parse_args()
     if args.impl == "reference":
-        if args.workload in DECODE_MODELS or args.workload in ("large_batch", "block"):
+        if args.workload in DECODE_MODELS or args.workload in ("large_batch", "block", "quantize"):
             raise SystemExit("the reference arm times the oracle on the layer workloads (config*, tiny, large)")
         run_reference(args)
     elif args.workload in DECODE_MODELS:
@@ -1039,6 +1174,8 @@ def main():
         run_large_batch(args)
     elif args.workload == "block":
         run_block(args)
+    elif args.workload == "quantize":
+        run_quantize(args)
     else:
         run_library(args)
 

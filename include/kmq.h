@@ -303,6 +303,74 @@ kmq_status kmq_block_dequant_to_bf16(const uint8_t* wq, const uint16_t* scales, 
                                      int64_t N, int64_t K, int bits, void* stream);
 
 /*
+ * The quantiser side: from float32 weights to codebooks, scales and packed
+ * indices (Section 2.1 "Rounding to nearest centroids", Eq. "centroid
+ * quantizer": f_c(x) = argmin_{c_i} |x - c_i|, the centroids "obtained
+ * algorithmically by 1D k-means clustering"; "Block formats"; Section 2.2: the
+ * scale functions absmax and absmean, "Nonlinear k-means quantization").  The
+ * value Q(w) that quantisation-aware training substitutes for w in the forward
+ * pass (Section 2.1, "Quantization-Aware Training") is what
+ * kmq_dequant_to_bf16 / kmq_block_dequant_to_bf16 return for the output of
+ * these calls.  Where the paper is silent the rules are: start at the 2^bits
+ * linearly interpolated quantiles (i + 1/2) / 2^bits of the values; `iters`
+ * Lloyd iterations (assign, then move each centroid to the float64 mean of its
+ * values; an empty cluster keeps its centroid); a value half-way between two
+ * centroids goes to the lower one; equal centroids are represented by the
+ * lowest index; the stored centroid is the float64 mean rounded to float32 and
+ * then to bf16, to nearest even, a zero of either sign as +0.  Weights must be
+ * finite.
+ *
+ * kmq_kmeans_rows -- one fit per row.
+ *   W          DEVICE float32 [N, K] row-major, read only.
+ *   bits       1, 2, 4 or 8 (8 for the shared codebook of the block format).
+ *   codebooks  DEVICE bf16 [N, 2^bits], non-decreasing along a row.
+ *   centroids  DEVICE float64 [N, 2^bits] or NULL: the unrounded centroids.
+ *   A row is sorted in shared memory: 2^bits <= K <= 32768, else KMQ_ERR_SHAPE.
+ * kmq_assign_pack -- packed[n, k] = index of the centroid of codebooks[n, :]
+ *   nearest to W[n, k], written directly in `layout` (the argument rules of
+ *   kmq_pack).  Codebook rows must be non-decreasing (otherwise the indices are
+ *   valid but need not be the nearest).  The decision is exact: no rounding is
+ *   involved in comparing a weight with the midpoint of two stored centroids.
+ * kmq_quantize_rows -- kmq_kmeans_rows, then kmq_assign_pack with the stored
+ *   codebooks, on one stream.
+ * kmq_block_scales -- scales[n, g] = bf16(lambda(W[n, 64g .. 64g+64))), lambda
+ *   = max |w| (KMQ_LAMBDA_ABSMAX) or mean |w| (KMQ_LAMBDA_ABSMEAN, the 64
+ *   magnitudes added in float64 in index order); a scale that would be stored
+ *   as zero is stored as 1.  K a multiple of 64.
+ * kmq_block_sample -- the normalised weights w / scale (float64 quotient with
+ *   the stored scale, not clipped: within [-1, 1] up to the rounding of an
+ *   absmax scale, beyond it under absmean) at the flat positions 0, s, 2s, ... with
+ *   s = max(1, N*K / samples), the first kmq_block_sample_count(N, K, samples)
+ *   of them, rounded to float32 into `out` (DEVICE): the values the shared
+ *   codebook is fitted on (kmq_kmeans_rows with N = 1, bits up to 8).
+ * kmq_block_assign_pack -- wq = the packed indices (layout of kmq_block_pack)
+ *   of the centroid of `codebook` (DEVICE bf16 [2^bits], non-decreasing)
+ *   nearest to each normalised weight.
+ * kmq_block_quantize -- the four steps above in order on one stream;
+ *   `sample_workspace` DEVICE float32 [samples], 2^bits <= samples <= 32768.
+ * All pointers 16-byte aligned.  Errors: KMQ_ERR_NULL, KMQ_ERR_BITS,
+ * KMQ_ERR_SHAPE, KMQ_ERR_ALIGN, KMQ_ERR_LAYOUT (unknown layout or lambda),
+ * KMQ_ERR_CUDA.
+ */
+#define KMQ_LAMBDA_ABSMAX 0
+#define KMQ_LAMBDA_ABSMEAN 1
+kmq_status kmq_kmeans_rows(const float* W, int64_t N, int64_t K, int bits, int iters, uint16_t* codebooks,
+                           double* centroids, void* stream);
+kmq_status kmq_assign_pack(const float* W, const uint16_t* codebooks, int64_t N, int64_t K, int bits, int layout,
+                           uint32_t* packed, void* stream);
+kmq_status kmq_quantize_rows(const float* W, int64_t N, int64_t K, int bits, int iters, int layout,
+                             uint16_t* codebooks, uint32_t* packed, void* stream);
+kmq_status kmq_block_scales(const float* W, int64_t N, int64_t K, int lambda, uint16_t* scales, void* stream);
+int64_t kmq_block_sample_count(int64_t N, int64_t K, int64_t samples);
+kmq_status kmq_block_sample(const float* W, const uint16_t* scales, int64_t N, int64_t K, int64_t samples, float* out,
+                            void* stream);
+kmq_status kmq_block_assign_pack(const float* W, const uint16_t* scales, const uint16_t* codebook, int64_t N,
+                                 int64_t K, int bits, uint8_t* wq, void* stream);
+kmq_status kmq_block_quantize(const float* W, int64_t N, int64_t K, int bits, int lambda, int iters, int64_t samples,
+                              uint16_t* scales, uint16_t* codebook, uint8_t* wq, float* sample_workspace,
+                              void* stream);
+
+/*
  * Measurement helpers (conveniences of this library; the paper has no
  * counterpart).  They put the layer's timings into proportion on the GPU at
  * hand:

@@ -25,10 +25,12 @@ What it leaves open, and the reading taken here (the same on both sides of every
   ``2x = s`` and ``e < 0`` (if ``2x`` differs from ``s`` it differs by more than ``|e|``, both being multiples of the
   last place of ``s`` or far apart);
 * arithmetic: float64 sums and means; the stored centroid is the float64 mean rounded to float32 and then to bf16,
-  both to nearest even;
+  both to nearest even; a centroid that is zero is stored as +0 (the sign of a zero mean depends on the order of
+  the additions and carries no information);
 * absmean sums the 64 magnitudes in float64 in index order (the order is part of the reading so that the stored bf16
-  scale is reproducible bit for bit); a block of zeros gets scale 1; normalised weight = ``clip(w / scale, -1, 1)``
-  in float64 with the stored scale;
+  scale is reproducible bit for bit); a block of zeros gets scale 1; normalised weight = ``w / scale``, the
+  float64 quotient with the stored scale, not clipped: with absmax it lies in [-1, 1] up to the bf16 rounding of the
+  scale (at most 1 + 2^-8 in magnitude), with absmean it does not, and the paper fits k-means under both;
 * the per-tensor fit of the block format runs on an evenly strided sample of the normalised weights, rounded to
   float32: flat indices ``0, s, 2s, ...`` with ``s = max(1, N*K // samples)``, the first ``samples`` of them.
 
@@ -118,8 +120,9 @@ def lloyd_rows(W: np.ndarray, bits: int, iters: int = 20) -> np.ndarray:
 
 
 def centroids_to_bf16(c: np.ndarray) -> np.ndarray:
-    """Stored form of fitted centroids: float64 -> float32 -> bf16, each step to nearest even."""
-    return f32_to_bf16_rne(np.asarray(c, dtype=np.float64).astype(np.float32))
+    """Stored form of fitted centroids: float64 -> float32 -> bf16, each step to nearest even; zero as +0."""
+    bits = f32_to_bf16_rne(np.asarray(c, dtype=np.float64).astype(np.float32))
+    return np.where((bits & np.uint16(0x7FFF)) == 0, np.uint16(0), bits).astype(np.uint16)
 
 
 def _first_of_equal(cb: np.ndarray) -> np.ndarray:
@@ -167,11 +170,11 @@ def block_scales(W: np.ndarray, mode: int = ABSMAX) -> np.ndarray:
 
 
 def normalise(W: np.ndarray, scales_bf16: np.ndarray) -> np.ndarray:
-    """clip(w / stored scale, -1, 1) in float64: [N, K]."""
+    """w / stored scale in float64: [N, K]."""
     W = np.asarray(W, dtype=np.float32)
     N, K = W.shape
     s = _bf16_to_f64(scales_bf16).reshape(N, K // BLOCK, 1)
-    return np.clip(W.astype(np.float64).reshape(N, K // BLOCK, BLOCK) / s, -1.0, 1.0).reshape(N, K)
+    return (W.astype(np.float64).reshape(N, K // BLOCK, BLOCK) / s).reshape(N, K)
 
 
 def strided_sample(W: np.ndarray, scales_bf16: np.ndarray, samples: int) -> np.ndarray:

@@ -22,6 +22,7 @@ KMQ_LAYOUT_CANONICAL = 0
 KMQ_LAYOUT_TUNED = 1
 KMQ_LAYOUT_TABLE = 2
 KMQ_SCALE_DIRECT, KMQ_SCALE_DEFERRED = 0, 1
+KMQ_LAMBDA_ABSMAX, KMQ_LAMBDA_ABSMEAN = 0, 1
 KMQ_DEVICE_ERROR_WAIT_TIMEOUT = 1
 KMQ_DEVICE_ERROR_SMEM_WINDOW = 2
 
@@ -52,6 +53,14 @@ SIGNATURES = {
     "kmq_block_pack": (_int, [_ptr, _i64, _i64, _int, _ptr, _ptr]),
     "kmq_block_linear": (_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr]),
     "kmq_block_dequant_to_bf16": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _ptr]),
+    "kmq_kmeans_rows": (_int, [_ptr, _i64, _i64, _int, _int, _ptr, _ptr, _ptr]),
+    "kmq_assign_pack": (_int, [_ptr, _ptr, _i64, _i64, _int, _int, _ptr, _ptr]),
+    "kmq_quantize_rows": (_int, [_ptr, _i64, _i64, _int, _int, _int, _ptr, _ptr, _ptr]),
+    "kmq_block_scales": (_int, [_ptr, _i64, _i64, _int, _ptr, _ptr]),
+    "kmq_block_sample_count": (_i64, [_i64, _i64, _i64]),
+    "kmq_block_sample": (_int, [_ptr, _ptr, _i64, _i64, _i64, _ptr, _ptr]),
+    "kmq_block_assign_pack": (_int, [_ptr, _ptr, _ptr, _i64, _i64, _int, _ptr, _ptr]),
+    "kmq_block_quantize": (_int, [_ptr, _i64, _i64, _int, _int, _int, _i64, _ptr, _ptr, _ptr, _ptr, _ptr]),
     "kmq_probe_launch": (_int, [_ptr]),
     "kmq_probe_read_out_bytes": (_sz, []),
     "kmq_probe_read": (_int, [_ptr, _sz, _ptr, _ptr]),
@@ -260,4 +269,64 @@ def kmq_block_dequant_to_bf16(wq, scales, codebook, W, N, K, bits, stream=None, 
                                          _stream(stream))
     if check:
         _check(st, "kmq_block_dequant_to_bf16")
+    return st
+
+
+def kmq_kmeans_rows(W, N, K, bits, iters, codebooks, centroids=None, stream=None, check=True) -> int:
+    """Per-row 1-D Lloyd fit: W float32 [N, K] -> codebooks bf16 [N, 2^bits] (and float64 centroids if given)."""
+    st = lib().kmq_kmeans_rows(_addr(W), N, K, bits, iters, _addr(codebooks), _addr(centroids), _stream(stream))
+    if check:
+        _check(st, "kmq_kmeans_rows")
+    return st
+
+
+def kmq_assign_pack(W, codebooks, N, K, bits, layout, packed, stream=None, check=True) -> int:
+    """Nearest stored centroid of every weight, written as packed indices in `layout`."""
+    st = lib().kmq_assign_pack(_addr(W), _addr(codebooks), N, K, bits, layout, _addr(packed), _stream(stream))
+    if check:
+        _check(st, "kmq_assign_pack")
+    return st
+
+
+def kmq_quantize_rows(W, N, K, bits, iters, layout, codebooks, packed, stream=None, check=True) -> int:
+    st = lib().kmq_quantize_rows(_addr(W), N, K, bits, iters, layout, _addr(codebooks), _addr(packed),
+                                 _stream(stream))
+    if check:
+        _check(st, "kmq_quantize_rows")
+    return st
+
+
+def kmq_block_scales(W, N, K, lam, scales, stream=None, check=True) -> int:
+    st = lib().kmq_block_scales(_addr(W), N, K, lam, _addr(scales), _stream(stream))
+    if check:
+        _check(st, "kmq_block_scales")
+    return st
+
+
+def kmq_block_sample_count(N, K, samples) -> int:
+    return lib().kmq_block_sample_count(N, K, samples)
+
+
+def kmq_block_sample(W, scales, N, K, samples, out, stream=None, check=True) -> int:
+    st = lib().kmq_block_sample(_addr(W), _addr(scales), N, K, samples, _addr(out), _stream(stream))
+    if check:
+        _check(st, "kmq_block_sample")
+    return st
+
+
+def kmq_block_assign_pack(W, scales, codebook, N, K, bits, wq, stream=None, check=True) -> int:
+    st = lib().kmq_block_assign_pack(_addr(W), _addr(scales), _addr(codebook), N, K, bits, _addr(wq),
+                                     _stream(stream))
+    if check:
+        _check(st, "kmq_block_assign_pack")
+    return st
+
+
+def kmq_block_quantize(W, N, K, bits, lam, iters, samples, scales, codebook, wq, sample_workspace, stream=None,
+                       check=True) -> int:
+    """Block format, all steps: scales, strided normalised sample, shared codebook fit, packed indices."""
+    st = lib().kmq_block_quantize(_addr(W), N, K, bits, lam, iters, samples, _addr(scales), _addr(codebook),
+                                  _addr(wq), _addr(sample_workspace), _stream(stream))
+    if check:
+        _check(st, "kmq_block_quantize")
     return st

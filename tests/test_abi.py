@@ -60,6 +60,14 @@ def test_sizes_and_strings():
     assert kmq.kmq_linear_variant(4096, 4096, 2, 1, layout=T) != kmq.kmq_linear_variant(4096, 4096, 2, 1)
 
 
+def test_block_sample_count():
+    assert kmq.kmq_block_sample_count(4, 128, 100) == 100          # stride 5: 103 positions, the first 100
+    assert kmq.kmq_block_sample_count(4, 128, 10 ** 6) == 512
+    assert kmq.kmq_block_sample_count(4, 128, 512) == 512
+    assert kmq.kmq_block_sample_count(4, 128, 300) == 300          # stride 1
+    assert kmq.kmq_block_sample_count(4, 100, 10) == 0             # K not a multiple of 64
+
+
 A = 0x1000  # a non-NULL, 16-byte aligned fake address; never dereferenced: validation fails first
 
 
@@ -85,6 +93,28 @@ A = 0x1000  # a non-NULL, 16-byte aligned fake address; never dereferenced: vali
     (lambda: kmq.kmq_dequant_to_bf16(A, 0, A, 4, 32, 1, stream=0, check=False), kmq.KMQ_ERR_NULL),
     (lambda: kmq.kmq_dequant_to_bf16(A, A, A, 4, 12, 4, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
     (lambda: kmq.kmq_dequant_to_bf16(A, A, A + 8, 4, 32, 1, stream=0, check=False), kmq.KMQ_ERR_ALIGN),
+    (lambda: kmq.kmq_kmeans_rows(0, 4, 64, 2, 20, A, stream=0, check=False), kmq.KMQ_ERR_NULL),
+    (lambda: kmq.kmq_kmeans_rows(A, 4, 64, 3, 20, A, stream=0, check=False), kmq.KMQ_ERR_BITS),
+    (lambda: kmq.kmq_kmeans_rows(A, 4, 32769, 2, 20, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
+    (lambda: kmq.kmq_kmeans_rows(A, 4, 8, 4, 20, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
+    (lambda: kmq.kmq_kmeans_rows(A, 4, 64, 2, -1, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
+    (lambda: kmq.kmq_kmeans_rows(A, 4, 64, 2, 20, A, A + 8, stream=0, check=False), kmq.KMQ_ERR_ALIGN),
+    (lambda: kmq.kmq_assign_pack(A, 0, 4, 32, 1, 0, A, stream=0, check=False), kmq.KMQ_ERR_NULL),
+    (lambda: kmq.kmq_assign_pack(A, A, 4, 32, 8, 0, A, stream=0, check=False), kmq.KMQ_ERR_BITS),
+    (lambda: kmq.kmq_assign_pack(A, A, 4, 24, 2, 0, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
+    (lambda: kmq.kmq_assign_pack(A, A, 4, 32, 1, 5, A, stream=0, check=False), kmq.KMQ_ERR_LAYOUT),
+    (lambda: kmq.kmq_assign_pack(A + 4, A, 4, 32, 1, 0, A, stream=0, check=False), kmq.KMQ_ERR_ALIGN),
+    (lambda: kmq.kmq_quantize_rows(A, 4, 65536, 1, 20, 0, A, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
+    (lambda: kmq.kmq_quantize_rows(A, 4, 64, 1, 20, 0, A, 0, stream=0, check=False), kmq.KMQ_ERR_NULL),
+    (lambda: kmq.kmq_block_scales(A, 4, 96, 0, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
+    (lambda: kmq.kmq_block_scales(A, 4, 128, 2, A, stream=0, check=False), kmq.KMQ_ERR_LAYOUT),
+    (lambda: kmq.kmq_block_scales(A, 4, 128, 0, 0, stream=0, check=False), kmq.KMQ_ERR_NULL),
+    (lambda: kmq.kmq_block_sample(A, A, 4, 128, 0, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
+    (lambda: kmq.kmq_block_assign_pack(A, A, A, 4, 128, 3, A, stream=0, check=False), kmq.KMQ_ERR_BITS),
+    (lambda: kmq.kmq_block_assign_pack(A, A, A + 2, 4, 128, 4, A, stream=0, check=False), kmq.KMQ_ERR_ALIGN),
+    (lambda: kmq.kmq_block_quantize(A, 4, 128, 4, 0, 20, 8, A, A, A, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
+    (lambda: kmq.kmq_block_quantize(A, 4, 128, 4, 0, 20, 40000, A, A, A, 0, stream=0, check=False), kmq.KMQ_ERR_NULL),
+    (lambda: kmq.kmq_block_quantize(A, 4096, 4096, 4, 0, 20, 40000, A, A, A, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
 ])
 def test_validation_status_codes(call, expected):
     assert call() == expected
