@@ -718,7 +718,14 @@ def run_quantize(args):
             stream.synchronize()
         return e0.elapsed_time(e1) / steps
 
-    for (fmt, N, K, bits) in QUANTIZE_CASES:
+    cases = QUANTIZE_CASES
+    if args.case:      # e.g. "format=rows,N=4096,bits=4": a subset small enough for a profiler run
+        want = dict(kv.split("=") for kv in args.case.split(","))
+        cases = [c for c in cases if all(str({"format": c[0], "N": c[1], "K": c[2], "bits": c[3]}[k]) == v
+                                         for k, v in want.items())]
+        if not cases:
+            raise SystemExit(f"--case {args.case!r} matches no case of the quantize workload")
+    for (fmt, N, K, bits) in cases:
         g = torch.Generator(device=dev).manual_seed(N + K + bits)
         pool = max(2, -(-(L2_BYTES + L2_BYTES // 2) // (N * K * 4)))
         W = torch.randn((pool, N, K), generator=g, device=dev, dtype=torch.float32) * 0.02
@@ -796,7 +803,7 @@ def run_quantize(args):
         "config": {"workload": "quantize: per-row 1-D Lloyd fit (quantile start, 20 iterations) + nearest-centroid "
                                "assignment + packing (kmq_quantize_rows), and the block format's scales + sampled "
                                "shared-codebook fit + assignment (kmq_block_quantize, absmax, 32768 samples), on "
-                               + str([(f, N, K, b) for (f, N, K, b) in QUANTIZE_CASES]) + ", N(0, 0.02) float32 weights",
+                               + str([(f, N, K, b) for (f, N, K, b) in cases]) + ", N(0, 0.02) float32 weights",
                    "l2": "inputs larger than L2: consecutive calls read different copies of the weights, pool >= 1.5 x 126 MB",
                    "multi_gpu": "replicas only"},
         "per_case": rows_out,

@@ -49,11 +49,10 @@ __global__ void __launch_bounds__(1024) lloyd_rows_kernel(const float* __restric
         for (int t = tid; t < (P >> 1); t += nthr) {
           const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1)), p = i | j;
           const uint32_t a = keys[i], b = keys[p];
+          const uint32_t lo = min(a, b), hi = max(a, b);
           const bool up = (i & k) == 0;
-          if ((a > b) == up) {
-            keys[i] = b;
-            keys[p] = a;
-          }
+          keys[i] = up ? lo : hi;
+          keys[p] = up ? hi : lo;
         }
         __syncthreads();
       }
@@ -177,8 +176,9 @@ __device__ __forceinline__ int count_below(double two_x, const Mid* mids) {
 
 constexpr int kLayoutCanonical = 0, kLayoutTuned = 1, kLayoutPlanes = 2;
 
-// One CTA per tile of 16 rows; the tile's midpoints and its lowest-equal-index maps sit in shared memory; a thread
-// builds one 32-bit word of the packed output from the float32 weights that word covers.
+// CTA (x, y) takes share y of the output words of tile x (16 rows); the tile's midpoints and its lowest-equal-index
+// maps sit in shared memory; a thread builds one 32-bit word of the packed output from the float32 weights that word
+// covers.
 template <int BITS, int LAYOUT>
 __global__ void __launch_bounds__(256) assign_pack_kernel(const float* __restrict__ W,
                                                           const uint16_t* __restrict__ codebooks,
@@ -221,7 +221,8 @@ __global__ void __launch_bounds__(256) assign_pack_kernel(const float* __restric
     const int64_t chunks = table_chunks(K);
     const int64_t words = chunks * BITS * 128;
     uint32_t* out = packed + tile * words;
-    for (int64_t l = threadIdx.x; l < words; l += blockDim.x) {
+    for (int64_t l = words * blockIdx.y / gridDim.y + threadIdx.x; l < words * (blockIdx.y + 1) / gridDim.y;
+         l += blockDim.x) {
       const int64_t unit = l >> 7;
       const int lane = (int)(l & 127) >> 2, q = (int)(l & 3);
       const int plane = (int)(unit % BITS);
@@ -247,7 +248,8 @@ __global__ void __launch_bounds__(256) assign_pack_kernel(const float* __restric
     constexpr bool TUNED = LAYOUT == kLayoutTuned;
     const int64_t steps = tuned_steps(wpr);
     const int64_t words = TUNED ? steps * 256 : 16 * wpr;
-    for (int64_t l = threadIdx.x; l < words; l += blockDim.x) {
+    for (int64_t l = words * blockIdx.y / gridDim.y + threadIdx.x; l < words * (blockIdx.y + 1) / gridDim.y;
+         l += blockDim.x) {
       int r;
       int64_t j;
       if constexpr (TUNED) {
@@ -380,11 +382,20 @@ inline int capped_grid(int64_t items, int threads, int sm_count, int per_sm) {
 template <int BITS>
 cudaError_t launch_assign_bits(const float* W, const uint16_t* cb, int64_t N, int64_t K, int layout, uint32_t* packed,
                                cudaStream_t s) {
-  const int tiles = (int)((N + 15) / 16);
-  if (layout == KMQ_LAYOUT_CANONICAL) assign_pack_kernel<BITS, kLayoutCanonical><<<tiles, 256, 0, s>>>(W, cb, packed, N, K);
+  const DeviceInfo* di = device_info();
+  if (!di) return cudaErrorInvalidDevice;
+  const int64_t tiles = (N + 15) / 16;
+  // enough CTAs to fill the machine several times over, each with at least a few words per thread
+  int64_t shares = ((int64_t)di->sm_count * 16 + tiles - 1) / tiles;
+  const int64_t max_shares = 16 * (K / (32 / BITS)) / 1024;
+  if (shares > max_shares) shares = max_shares;
+  if (shares < 1) shares = 1;
+  if (shares > 65535) shares = 65535;
+  const dim3 grid((unsigned)tiles, (unsigned)shares);
+  if (layout == KMQ_LAYOUT_CANONICAL) assign_pack_kernel<BITS, kLayoutCanonical><<<grid, 256, 0, s>>>(W, cb, packed, N, K);
   else if (layout == KMQ_LAYOUT_TABLE && BITS != 4)
-    assign_pack_kernel<BITS == 4 ? 1 : BITS, kLayoutPlanes><<<tiles, 256, 0, s>>>(W, cb, packed, N, K);
-  else assign_pack_kernel<BITS, kLayoutTuned><<<tiles, 256, 0, s>>>(W, cb, packed, N, K);
+    assign_pack_kernel<BITS == 4 ? 1 : BITS, kLayoutPlanes><<<grid, 256, 0, s>>>(W, cb, packed, N, K);
+  else assign_pack_kernel<BITS, kLayoutTuned><<<grid, 256, 0, s>>>(W, cb, packed, N, K);
   return cudaGetLastError();
 }
 
