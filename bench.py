@@ -571,7 +571,7 @@ def run_large_batch(args):
 # --------------------------------------------------------------------------
 # the paper's own block format (shared codebook + bf16 scale per block of 64)
 # --------------------------------------------------------------------------
-BLOCK_CASES = [(4096, 4096, b, 1) for b in (1, 2, 4, 8)] + [(8192, 8192, b, 1) for b in (1, 4)]
+BLOCK_CASES = [(4096, 4096, b, 1) for b in (1, 2, 4, 8)] + [(8192, 8192, b, 1) for b in (1, 2, 4)]
 
 
 def block_bytes(N, K, bits, M):
@@ -639,14 +639,55 @@ def run_block(args):
             sampler.active = False
         us = e0.elapsed_time(e1) * 1e3 / (steps * pool)
         launches += steps * pool
+        us_table = None
+        if bits != 8:
+            # the same layers through the activation-table kernel, which reads its own layout (index bytes and
+            # scales side by side): packed once, outside the timed region
+            tab = torch.empty((pool, kmq.kmq_block_table_bytes(N, K, bits)), dtype=torch.uint8, device=dev)
+            kmq.kmq_block_table_pack(wq[0], scales.view(torch.int16), N, K, bits, tab[0])
+            tab[1:] = tab[0]
+            wsb = kmq.kmq_block_table_workspace_bytes(N, K, bits)
+            ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device=dev)
+            y_t = torch.zeros(pool, M, N, dtype=torch.bfloat16, device=dev)
+
+            def call_t(i):
+                kmq.kmq_block_table_linear(tab[i], cb, x[i], y_t[i], N, K, bits, M, ws, wsb)
+            with torch.cuda.stream(stream):
+                call_t(0)
+                stream.synchronize()
+                gt = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gt, stream=stream):
+                    for i in range(pool):
+                        call_t(i)
+                for _ in range(max(args.warmup, 3)):
+                    gt.replay()
+                t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                sampler.active = True
+                t0.record(stream)
+                for _ in range(steps):
+                    gt.replay()
+                t1.record(stream)
+                stream.synchronize()
+                sampler.active = False
+            us_table = t0.elapsed_time(t1) * 1e3 / (steps * pool)
+            launches += steps * pool * (2 if wsb else 1)
         for i in (0, pool - 1):
             y_ref, s_abs = blk.block_linear_f64(ref_wq, scales.view(torch.int16).cpu().numpy().view(np.uint16)[rows],
                                                 cb.view(torch.int16).cpu().numpy().view(np.uint16),
                                                 x[i].view(torch.int16).cpu().numpy().view(np.uint16), K, bits)
             got = y[i][:, torch.from_numpy(rows).to(dev)].view(torch.int16).cpu().numpy().view(np.uint16)
             worst = max(worst, orc.check_linear(got, y_ref, s_abs))
+            if us_table is not None:
+                got = y_t[i][:, torch.from_numpy(rows).to(dev)].view(torch.int16).cpu().numpy().view(np.uint16)
+                worst = max(worst, orc.check_linear(got, y_ref, s_abs))
+        us_direct = us
+        if us_table is not None:
+            del tab, y_t
+            us = min(us, us_table)
         gbs = nbytes / us / 1e3
         rows_out.append({"N": N, "K": K, "bits": bits, "P_w": bits + 0.25, "M": M, "pool": pool, "us_per_call": round(us, 3),
+                         "us_kmq_block_linear": round(us_direct, 3),
+                         "us_kmq_block_table_linear": None if us_table is None else round(us_table, 3),
                          "gbs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peak_gbs, 4), "bytes_per_call": nbytes,
                          "ideal_us_at_measured_hbm": round(nbytes / (peak_gbs * 1e3), 3)})
         del wq, x, y
@@ -661,12 +702,13 @@ def run_block(args):
         "warmup": max(args.warmup, 3), "ms_per_step": round(tot_us * 1e-3, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "block: the paper's k-means block format (shared codebook, bf16 scale per block of 64, "
-                               "P_w = b + 0.25), kmq_block_linear with deferred scaling at batch 1 on "
+                               "P_w = b + 0.25), kmq_block_linear (deferred scaling) and kmq_block_table_linear at batch 1, the "
+                               "faster of the two per case, on "
                                + str([(N, K, b) for (N, K, b, _m) in BLOCK_CASES]) + ", random indices and scales",
                    "l2": "inputs larger than L2: every call of a step uses its own weight set, pool >= 2 x 126 MB",
                    "multi_gpu": "replicas only"},
         "per_case": rows_out,
-        "roofline": {"bound": "hbm", "kernel": f"kmq_block_linear b={dom['bits']} {dom['N']}x{dom['K']}",
+        "roofline": {"bound": "hbm", "kernel": f"block format b={dom['bits']} {dom['N']}x{dom['K']}",
                      "achieved": dom["gbs"], "peak": peak_gbs, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                      "frac": dom["frac_of_measured_hbm"], "traffic": None},
         "gpu_launches": launches, "clocks": sampler.summary(),

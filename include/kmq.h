@@ -303,6 +303,53 @@ kmq_status kmq_block_dequant_to_bf16(const uint8_t* wq, const uint16_t* scales, 
                                      int64_t N, int64_t K, int bits, void* stream);
 
 /*
+ * The block format through an activation table (b = 1, 2, 4; decode batches).
+ * With one codebook for the whole tensor, a 256-entry table per byte of packed
+ * indices can hold finished partial dot products of the activations with the
+ * centroids (the byte table of the paper's listing, Appendix "Benchmarking",
+ * "Kernel implementations", built over x instead of over the weights); the layer
+ * is then one shared-memory lookup per byte of weights and one multiply-add per
+ * block (deferred scaling).  The kernel reads its own layout, which holds the
+ * index bytes and the block scales of 16 rows x 32 bytes side by side:
+ *   unit (tile T = n / 16, chunk c = byte / 32) at byte offset
+ *   (T * chunks + c) * (512 + 32 * (4 / bits)),  chunks = ceil(K * bits / 256);
+ *   512 index bytes, then the bf16 scales scale[row r][block q of the chunk] at
+ *   512 + (r * (4 / bits) + q) * 2.  Lane L = 2 r + a owns the index bytes
+ *   [16 L, 16 L + 16); with S = 4 * bits, r = r_hi * S + r_lo, byte i = S * j + f
+ *   of the lane holds byte number
+ *   (8 * bits) * ((j + r_hi) % (4 / bits)) + a + 2 * ((f + r_lo) % S)
+ *   of the chunk of row 16 T + r.  Padding (rows >= N, bytes beyond K) is zero.
+ * kmq_block_table_bytes -- size of the table layout (0 for invalid arguments).
+ * kmq_block_table_index_offset / _scale_offset -- byte offset of the byte that
+ *   holds the index of weight (n, k), and of the scale of its block (-1 for
+ *   invalid arguments): the layout above as a function, for tools and tests.
+ * kmq_block_table_pack -- (wq, scales) of kmq_block_pack's layout -> table.
+ * kmq_block_table_unpack -- the inverse.
+ * kmq_block_table_workspace_bytes -- scratch kmq_block_table_linear needs for
+ *   this shape (0 when every CTA sees the whole of K).
+ * kmq_block_table_linear -- y[m, n] = sum_k x[m, k] * scale[n, k/64] *
+ *   c[idx[n, k]]: fp32 tables, fp32 accumulation, bf16 result, the tolerance
+ *   stated for kmq_linear for any finite codebook (a table entry is the sum of
+ *   the selected products themselves).  One pass over the weights per batch
+ *   row: meant for M = 1 .. 4.  Two launches per pass when scratch is needed.
+ *   Waits on copies are bounded; a run-out is reported by
+ *   kmq_device_error_flags only.  Needs 227 KB of shared memory per CTA
+ *   (KMQ_ERR_CUDA otherwise).
+ * bits = 1, 2 or 4 (KMQ_ERR_BITS), K a multiple of 64, pointers 16-byte aligned.
+ */
+size_t kmq_block_table_bytes(int64_t N, int64_t K, int bits);
+int64_t kmq_block_table_index_offset(int64_t n, int64_t k, int64_t N, int64_t K, int bits);
+int64_t kmq_block_table_scale_offset(int64_t n, int64_t k, int64_t N, int64_t K, int bits);
+kmq_status kmq_block_table_pack(const uint8_t* wq, const uint16_t* scales, int64_t N, int64_t K, int bits,
+                                uint8_t* table, void* stream);
+kmq_status kmq_block_table_unpack(const uint8_t* table, int64_t N, int64_t K, int bits, uint8_t* wq, uint16_t* scales,
+                                  void* stream);
+size_t kmq_block_table_workspace_bytes(int64_t N, int64_t K, int bits);
+kmq_status kmq_block_table_linear(const uint8_t* table, const uint16_t* codebook, const uint16_t* x, uint16_t* y,
+                                  int64_t N, int64_t K, int bits, int64_t M, void* workspace, size_t workspace_bytes,
+                                  void* stream);
+
+/*
  * The quantiser side: from float32 weights to codebooks, scales and packed
  * indices (Section 2.1 "Rounding to nearest centroids", Eq. "centroid
  * quantizer": f_c(x) = argmin_{c_i} |x - c_i|, the centroids "obtained

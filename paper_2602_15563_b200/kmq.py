@@ -53,6 +53,13 @@ SIGNATURES = {
     "kmq_block_pack": (_int, [_ptr, _i64, _i64, _int, _ptr, _ptr]),
     "kmq_block_linear": (_int, [_ptr, _ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _int, _ptr]),
     "kmq_block_dequant_to_bf16": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _ptr]),
+    "kmq_block_table_bytes": (_sz, [_i64, _i64, _int]),
+    "kmq_block_table_index_offset": (_i64, [_i64, _i64, _i64, _i64, _int]),
+    "kmq_block_table_scale_offset": (_i64, [_i64, _i64, _i64, _i64, _int]),
+    "kmq_block_table_pack": (_int, [_ptr, _ptr, _i64, _i64, _int, _ptr, _ptr]),
+    "kmq_block_table_unpack": (_int, [_ptr, _i64, _i64, _int, _ptr, _ptr, _ptr]),
+    "kmq_block_table_workspace_bytes": (_sz, [_i64, _i64, _int]),
+    "kmq_block_table_linear": (_int, [_ptr, _ptr, _ptr, _ptr, _i64, _i64, _int, _i64, _ptr, _sz, _ptr]),
     "kmq_kmeans_rows": (_int, [_ptr, _i64, _i64, _int, _int, _ptr, _ptr, _ptr]),
     "kmq_assign_pack": (_int, [_ptr, _ptr, _i64, _i64, _int, _int, _ptr, _ptr]),
     "kmq_quantize_rows": (_int, [_ptr, _i64, _i64, _int, _int, _int, _ptr, _ptr, _ptr]),
@@ -329,4 +336,44 @@ def kmq_block_quantize(W, N, K, bits, lam, iters, samples, scales, codebook, wq,
                                   _addr(wq), _addr(sample_workspace), _stream(stream))
     if check:
         _check(st, "kmq_block_quantize")
+    return st
+
+
+def kmq_block_table_bytes(N, K, bits) -> int:
+    return lib().kmq_block_table_bytes(N, K, bits)
+
+
+def kmq_block_table_index_offset(n, k, N, K, bits) -> int:
+    return lib().kmq_block_table_index_offset(n, k, N, K, bits)
+
+
+def kmq_block_table_scale_offset(n, k, N, K, bits) -> int:
+    return lib().kmq_block_table_scale_offset(n, k, N, K, bits)
+
+
+def kmq_block_table_pack(wq, scales, N, K, bits, table, stream=None, check=True) -> int:
+    st = lib().kmq_block_table_pack(_addr(wq), _addr(scales), N, K, bits, _addr(table), _stream(stream))
+    if check:
+        _check(st, "kmq_block_table_pack")
+    return st
+
+
+def kmq_block_table_unpack(table, N, K, bits, wq, scales, stream=None, check=True) -> int:
+    st = lib().kmq_block_table_unpack(_addr(table), N, K, bits, _addr(wq), _addr(scales), _stream(stream))
+    if check:
+        _check(st, "kmq_block_table_unpack")
+    return st
+
+
+def kmq_block_table_workspace_bytes(N, K, bits) -> int:
+    return lib().kmq_block_table_workspace_bytes(N, K, bits)
+
+
+def kmq_block_table_linear(table, codebook, x, y, N, K, bits, M, workspace=None, workspace_bytes=0, stream=None,
+                           check=True) -> int:
+    """Block format through the activation table: y = x * W^T, one pass per batch row."""
+    st = lib().kmq_block_table_linear(_addr(table), _addr(codebook), _addr(x), _addr(y), N, K, bits, M,
+                                      _addr(workspace), workspace_bytes, _stream(stream))
+    if check:
+        _check(st, "kmq_block_table_linear")
     return st

@@ -118,3 +118,39 @@ def table_from_indices(idx: np.ndarray, bits: int) -> np.ndarray:
         off = ((n // 16 * chunks + g // 32) * bits + p) * 512 + (2 * (n % 16) + g % 2) * 16 + ((g % 32) // 2 - n % 16) % 16
         out[off] = byte
     return out
+
+
+def block_table_from_bytes(wq: np.ndarray, scales: np.ndarray, K: int, bits: int) -> np.ndarray:
+    """The block-format table layout restated from the formulas of include/kmq.h: uint8 [total bytes].
+    wq uint8 [N, K*bits/8] (layout of kmq_block_pack), scales uint16 [N, K/64]."""
+    N = wq.shape[0]
+    bpc, S = 4 // bits, 4 * bits
+    unit = 512 + 32 * bpc
+    row_bytes, row_blocks = K * bits // 8, K // 64
+    chunks = -(-row_bytes // 32)
+    tiles = -(-N // 16)
+    out = np.zeros(tiles * chunks * unit, dtype=np.uint8)
+    sc = np.zeros(tiles * chunks * unit // 2, dtype=np.uint16)
+    for T in range(tiles):
+        for c in range(chunks):
+            base = (T * chunks + c) * unit
+            for r in range(16):
+                n = 16 * T + r
+                if n >= N:
+                    continue
+                r_hi, r_lo = divmod(r, S)
+                for a in range(2):
+                    L = 2 * r + a
+                    for i in range(16):
+                        j, f = divmod(i, S)
+                        byte = c * 32 + (8 * bits) * ((j + r_hi) % bpc) + a + 2 * ((f + r_lo) % S)
+                        if byte < row_bytes:
+                            out[base + 16 * L + i] = wq[n, byte]
+                for q in range(bpc):
+                    blk = c * bpc + q
+                    if blk < row_blocks:
+                        sc[(base + 512) // 2 + r * bpc + q] = scales[n, blk]
+    scb = sc.view(np.uint8)
+    mask = scb != 0
+    out[mask] = scb[mask]
+    return out

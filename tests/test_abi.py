@@ -93,6 +93,14 @@ A = 0x1000  # a non-NULL, 16-byte aligned fake address; never dereferenced: vali
     (lambda: kmq.kmq_dequant_to_bf16(A, 0, A, 4, 32, 1, stream=0, check=False), kmq.KMQ_ERR_NULL),
     (lambda: kmq.kmq_dequant_to_bf16(A, A, A, 4, 12, 4, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
     (lambda: kmq.kmq_dequant_to_bf16(A, A, A + 8, 4, 32, 1, stream=0, check=False), kmq.KMQ_ERR_ALIGN),
+    (lambda: kmq.kmq_block_table_pack(A, 0, 4, 128, 1, A, stream=0, check=False), kmq.KMQ_ERR_NULL),
+    (lambda: kmq.kmq_block_table_pack(A, A, 4, 128, 8, A, stream=0, check=False), kmq.KMQ_ERR_BITS),
+    (lambda: kmq.kmq_block_table_pack(A, A, 4, 96, 2, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
+    (lambda: kmq.kmq_block_table_unpack(A, 4, 128, 2, A, A + 2, stream=0, check=False), kmq.KMQ_ERR_ALIGN),
+    (lambda: kmq.kmq_block_table_linear(A, A, A, 0, 4, 128, 1, 1, stream=0, check=False), kmq.KMQ_ERR_NULL),
+    (lambda: kmq.kmq_block_table_linear(A, A, A, A, 4, 128, 3, 1, stream=0, check=False), kmq.KMQ_ERR_BITS),
+    (lambda: kmq.kmq_block_table_linear(A, A, A, A, 4, 128, 1, 0, stream=0, check=False), kmq.KMQ_ERR_SHAPE),
+    (lambda: kmq.kmq_block_table_linear(A, A + 8, A, A, 4, 128, 1, 1, stream=0, check=False), kmq.KMQ_ERR_ALIGN),
     (lambda: kmq.kmq_kmeans_rows(0, 4, 64, 2, 20, A, stream=0, check=False), kmq.KMQ_ERR_NULL),
     (lambda: kmq.kmq_kmeans_rows(A, 4, 64, 3, 20, A, stream=0, check=False), kmq.KMQ_ERR_BITS),
     (lambda: kmq.kmq_kmeans_rows(A, 4, 32769, 2, 20, A, stream=0, check=False), kmq.KMQ_ERR_SHAPE),

@@ -93,3 +93,39 @@ def test_bit_index_agrees_with_word_index_and_shift(bits):
                 for p in range(bits):
                     assert kmq.kmq_packed_bit_index(n, k, p, N, K, bits, layout) == w * 32 + sh + p
     assert kmq.kmq_packed_bytes(N, K, 4, kmq.KMQ_LAYOUT_TABLE) == kmq.kmq_packed_bytes(N, K, 4, T)
+
+
+@pytest.mark.parametrize("bits", (1, 2, 4))
+@pytest.mark.parametrize("N,K", ((16, 256), (37, 64 * 7), (5, 1024)))
+def test_block_table_offsets_are_injective_and_documented(bits, N, K):
+    """kmq_block_table_index_offset / _scale_offset against the layout of include/kmq.h restated here."""
+    bpc, S = 4 // bits, 4 * bits
+    unit = 512 + 32 * bpc
+    per = 8 // bits
+    chunks = -(-(K * bits // 8) // 32)
+    total = kmq.kmq_block_table_bytes(N, K, bits)
+    assert total == -(-N // 16) * chunks * unit
+    seen = set()
+    for n in range(N):
+        for k in range(0, K, per):
+            byte = k // per
+            c, b = divmod(byte, 32)
+            q, w = divmod(b, 8 * bits)
+            a, m = w & 1, w >> 1
+            r = n % 16
+            r_hi, r_lo = divmod(r, S)
+            j, f = (q - r_hi) % bpc, (m - r_lo) % S
+            want = ((n // 16) * chunks + c) * unit + 16 * (2 * r + a) + S * j + f
+            got = kmq.kmq_block_table_index_offset(n, k, N, K, bits)
+            assert got == want == kmq.kmq_block_table_index_offset(n, k + per - 1, N, K, bits)
+            assert got % unit < 512 and got not in seen
+            seen.add(got)
+        for blk in range(K // 64):
+            want = ((n // 16) * chunks + blk // bpc) * unit + 512 + ((n % 16) * bpc + blk % bpc) * 2
+            got = kmq.kmq_block_table_scale_offset(n, 64 * blk + 63, N, K, bits)
+            assert got == want and got not in seen and got + 1 not in seen
+            seen.update((got, got + 1))
+    assert max(seen) < total
+    assert kmq.kmq_block_table_index_offset(N, 0, N, K, bits) == -1
+    assert kmq.kmq_block_table_scale_offset(0, K, N, K, bits) == -1
+    assert kmq.kmq_block_table_bytes(N, K, 8) == 0 and kmq.kmq_block_table_bytes(N, K + 32, bits) == 0
