@@ -602,7 +602,14 @@ def run_block(args):
     stream = torch.cuda.Stream()
     steps = max(1, min(args.steps, 50))
     rows_out, launches, worst = [], 0, 0.0
-    for (N, K, bits, M) in BLOCK_CASES:
+    cases = BLOCK_CASES
+    if args.case:      # e.g. "N=8192,bits=1": one case, small enough for a profiler run
+        want = dict(kv.split("=") for kv in args.case.split(","))
+        cases = [c for c in cases if all(str({"N": c[0], "K": c[1], "bits": c[2], "M": c[3]}[k]) == v
+                                         for k, v in want.items())]
+        if not cases:
+            raise SystemExit(f"--case {args.case!r} matches no case of the block workload")
+    for (N, K, bits, M) in cases:
         g = torch.Generator(device=dev).manual_seed(N + 7 * bits)
         nbytes = block_bytes(N, K, bits, M)
         pool = max(4, -(-2 * L2_BYTES // nbytes))
@@ -704,7 +711,7 @@ def run_block(args):
         "config": {"workload": "block: the paper's k-means block format (shared codebook, bf16 scale per block of 64, "
                                "P_w = b + 0.25), kmq_block_linear (deferred scaling) and kmq_block_table_linear at batch 1, the "
                                "faster of the two per case, on "
-                               + str([(N, K, b) for (N, K, b, _m) in BLOCK_CASES]) + ", random indices and scales",
+                               + str([(N, K, b) for (N, K, b, _m) in cases]) + ", random indices and scales",
                    "l2": "inputs larger than L2: every call of a step uses its own weight set, pool >= 2 x 126 MB",
                    "multi_gpu": "replicas only"},
         "per_case": rows_out,
