@@ -25,9 +25,11 @@
 // bulk asynchronous copies (cp.async.bulk, completion on an mbarrier per stage): no registers and no scoreboard
 // slots are tied up by loads in flight, so up to 32 warps of 64 registers run per SM.  A lane owns one row of the
 // tile and every second group, keeps its running sums in registers over the NL chunks and adds the two lanes of a row
-// with one shuffle.  With a single slice the warp applies the codebook and stores its rows directly; otherwise the
-// per-slice sums go to scratch [slice][class][row] and a second kernel adds the slices in a fixed order, applies the
-// codebook and stores bf16.
+// with one shuffle.  With a single slice the warp applies the codebook and stores its rows directly.  With 2, 4 or 8
+// slices that fit the machine as thread-block clusters, the slices of a row block are one cluster: the sums stay in
+// each CTA's shared memory and, after a cluster barrier, CTA s adds its share of the rows over all slices out of the
+// other CTAs' shared memory (fixed order), applies the codebook and stores.  Otherwise the per-slice sums go to
+// scratch [slice][class][row] and a second kernel adds the slices in a fixed order, applies the codebook and stores.
 //
 // Programmatic dependent launch: the CTA may start while the previous kernel on the stream is still running.  Until
 // griddepcontrol.wait returns it only sets up its barriers, starts the first copies of packed indices (constants of
@@ -61,12 +63,29 @@ struct LutGeo {
   static constexpr uint32_t kBarBase = 1216;                             // mbarriers: 8 bytes per warp and stage
   static constexpr uint32_t kLowBase = 2304;                             // low stages: [kLowBase, kLutTableBase)
   static constexpr uint32_t kHighEnd = kTableEnd + (uint32_t)(kWarps * kStagesHigh * kPieceBytes);
+  // cluster variant: the CTA's partial sums [class][row of the block] sit between the low stages and the tables
+  static constexpr uint32_t kPartBase = kLowBase + (uint32_t)(kWarps * kStagesLow * kPieceBytes);
+  static constexpr int kPartFloats = (int)(kLutTableBase - kPartBase) / 4;
+  static constexpr uint32_t kSxWord = kSumBase + 40;                     // a free word of the sum area: sum of x
   static_assert(kBarBase + kWarps * kStages * 8 <= kLowBase, "mbarriers must fit below the low stages");
   static_assert(kLowBase + kWarps * kStagesLow * kPieceBytes <= kLutTableBase, "low stages overlap the tables");
   static_assert(kHighEnd <= 227 * 1024 + 1024, "stages exceed the shared memory of an SM");
   static_assert(NL >= 1 && NL <= 4 && (BITS == 1 || NL <= 3), "unsupported slice length");
   static_assert(kStages % kPieces == 0, "the ring must hold whole tiles");
 };
+
+// ---- thread-block cluster: barrier and loads from another CTA's shared memory ----
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// `saddr`: an address in this CTA's shared-memory window; the value at the same place of the CTA of rank `rank`.
+__device__ __forceinline__ float ld_cluster_f32(uint32_t saddr, uint32_t rank) {
+  uint32_t ra;
+  float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(saddr), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+  return v;
+}
 
 // Index of the centroid of smallest magnitude (lowest index on ties); `c` = the row's codebook as bf16 pairs.
 template <int BITS>
@@ -107,7 +126,7 @@ template <int BITS, int NL>
 __global__ void __launch_bounds__(LutGeo<BITS, NL>::kWarps * 32, 1)
     linear_lut_kernel(const unsigned char* __restrict__ packed, const uint16_t* __restrict__ cb,
                       const uint16_t* __restrict__ x, uint16_t* __restrict__ y, float* __restrict__ scratch, int64_t N,
-                      int64_t K, int slices, int row_blocks, unsigned int* __restrict__ err) {
+                      int64_t K, int slices, int row_blocks, unsigned int* __restrict__ err, int in_cluster) {
   using G = LutGeo<BITS, NL>;
   constexpr int CL = G::kClasses, S = G::kStages, P = G::kPieces, PC = G::kPieceChunks, TPR = G::kTasksPerRound;
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -121,14 +140,19 @@ __global__ void __launch_bounds__(LutGeo<BITS, NL>::kWarps * 32, 1)
   const int64_t rows_pad = (int64_t)tiles * 16;
   const int chunk0 = slice * NL;
   const int t0 = (int)((int64_t)tiles * rb / row_blocks), t1 = (int)((int64_t)tiles * (rb + 1) / row_blocks);
+  const int rows_blk = (t1 - t0) * 16;   // rows of this row block, padding included
 
   // Tables, stages and barriers sit at absolute shared-memory addresses: the dynamic shared memory of this CTA must
   // cover [kSumBase, kHighEnd).
+  // In a cluster launch the shared-memory window of the CTA of rank r starts at r << 24 of the shared address space
+  // (0 without a cluster); every absolute address below carries this base.  It leaves bits 8..15 alone, which the
+  // lookups overwrite with the table entry.
+  const uint32_t wb = smem_addr(smem_raw) & 0xFF000000u;
   {
-    const uint32_t s0 = smem_addr(smem_raw);
+    const uint32_t s0 = smem_addr(smem_raw) - wb;
     uint32_t dyn;
     asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
-    if (s0 > G::kSumBase || s0 + dyn < G::kHighEnd) {
+    if (s0 > G::kSumBase || s0 + dyn < G::kHighEnd) {   // the same in every CTA of the grid: all of them leave here
       asm volatile("griddepcontrol.wait;" ::: "memory");
       if (threadIdx.x == 0) atomicOr(err, kErrWindow);
       return;
@@ -137,9 +161,9 @@ __global__ void __launch_bounds__(LutGeo<BITS, NL>::kWarps * 32, 1)
 
   // ---- this warp's ring: stage st < kStagesHigh above the tables, the others below.  Stage tt * P + pc holds
   //      piece pc of the warp's tile number ti with ti % TPR = tt; round number ti / TPR gives the mbarrier phase ----
-  const uint32_t bar0 = G::kBarBase + (uint32_t)(warp * S) * 8u;
-  const uint32_t high0 = G::kTableEnd + (uint32_t)(warp * G::kStagesHigh * G::kPieceBytes);
-  const uint32_t low0 = G::kLowBase + (uint32_t)(warp * G::kStagesLow * G::kPieceBytes);
+  const uint32_t bar0 = wb + G::kBarBase + (uint32_t)(warp * S) * 8u;
+  const uint32_t high0 = wb + G::kTableEnd + (uint32_t)(warp * G::kStagesHigh * G::kPieceBytes);
+  const uint32_t low0 = wb + G::kLowBase + (uint32_t)(warp * G::kStagesLow * G::kPieceBytes);
   auto stage_addr = [&](int st) -> uint32_t {   // st is a compile-time constant wherever this is called
     return st < G::kStagesHigh ? high0 + (uint32_t)(st * G::kPieceBytes)
                                : low0 + (uint32_t)((st - G::kStagesHigh) * G::kPieceBytes);
@@ -186,7 +210,7 @@ __global__ void __launch_bounds__(LutGeo<BITS, NL>::kWarps * 32, 1)
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
       // through an opaque move: the 16 values must stay in registers
-      asm volatile("mov.u32 %0, %1;" : "=r"(base[i]) : "r"(kLutTableBase | ((uint32_t)(a + 2 * ((r + i) & 15)) << 2)));
+      asm volatile("mov.u32 %0, %1;" : "=r"(base[i]) : "r"(wb | kLutTableBase | ((uint32_t)(a + 2 * ((r + i) & 15)) << 2)));
     }
   }
   auto row_codebook = [&](int ti, uint32_t (&c)[2]) {   // codebook of this lane's row of the warp's tile number ti
@@ -232,7 +256,7 @@ __global__ void __launch_bounds__(LutGeo<BITS, NL>::kWarps * 32, 1)
         l[4] = x2;   l[5] = x0 + x2;  l[6] = x1 + x2;  l[7] = l[3] + x2;
 #pragma unroll
         for (int i = 0; i < 8; ++i) l[8 + i] = l[i] + x3;
-        const uint32_t dst = kLutTableBase + lut_slot_offset(j) + (uint32_t)h * 16u * 256u + (uint32_t)lane * 4u;
+        const uint32_t dst = wb + kLutTableBase + lut_slot_offset(j) + (uint32_t)h * 16u * 256u + (uint32_t)lane * 4u;
 #pragma unroll
         for (int i = 0; i < 16; ++i) sts_f32(dst + i * 256, l[i] + hs);
         // entry 255 = the sum of all 8 inputs of the group: summed over the chunk's groups by the warp of item (j, 15)
@@ -240,7 +264,7 @@ __global__ void __launch_bounds__(LutGeo<BITS, NL>::kWarps * 32, 1)
           float v = l[15] + hs;
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-          if (lane == 0) sts_f32(G::kSumBase + 4 * j, v);
+          if (lane == 0) sts_f32(wb + G::kSumBase + 4 * j, v);
         }
       }
     }
@@ -248,8 +272,11 @@ __global__ void __launch_bounds__(LutGeo<BITS, NL>::kWarps * 32, 1)
   __syncthreads();
   float sx_slice = 0.f;   // sum of the activations of this slice, chunk by chunk
 #pragma unroll
-  for (int j = 0; j < NL; ++j) sx_slice += lds_f32<0>(G::kSumBase + 4 * j);
-  if (threadIdx.x == 0 && slices > 1 && rb == 0) scratch[(size_t)slices * CL * rows_pad + slice] = sx_slice;
+  for (int j = 0; j < NL; ++j) sx_slice += lds_f32<0>(wb + G::kSumBase + 4 * j);
+  if (threadIdx.x == 0 && slices > 1) {
+    if (in_cluster) sts_f32(wb + G::kSxWord, sx_slice);
+    else if (rb == 0) scratch[(size_t)slices * CL * rows_pad + slice] = sx_slice;
+  }
 
   bool ok = true;
   for (int ti0 = 0; ti0 < my_tiles && ok; ti0 += TPR) {
@@ -320,6 +347,14 @@ __global__ void __launch_bounds__(LutGeo<BITS, NL>::kWarps * 32, 1)
             for (int q = 0; q < CL; ++q) out = fmaf(cent(s ^ (q + 1)) - cs, v[q], out);
             y[n] = (uint16_t)float_to_bf16_bits(out);
           }
+        } else if (in_cluster) {
+          // this CTA's share of the rows' sums stays in its shared memory for the reduction over the cluster
+          if ((lane & 1) == 0) {
+            const int row_local = (tile - t0) * 16 + (lane >> 1);
+#pragma unroll
+            for (int q = 0; q < CL; ++q)
+              sts_f32(wb + G::kPartBase + 4u * (uint32_t)(q * rows_blk + row_local), ok ? v[q] : 0.f);
+          }
         } else if (ok && (lane & 1) == 0) {
 #pragma unroll
           for (int q = 0; q < CL; ++q) part[(size_t)q * rows_pad] = v[q];
@@ -337,6 +372,44 @@ __global__ void __launch_bounds__(LutGeo<BITS, NL>::kWarps * 32, 1)
       if (!mbar_try(bar0 + 8 * st, 0)) (void)mbar_wait_slow(bar0 + 8 * st, 1);
     }
   }
+  if (!in_cluster) return;
+
+  // ---- reduction over the cluster: the `slices` CTAs of a row block are one thread-block cluster (rank = slice:
+  //      the grid is slice-major in x and the cluster spans `slices` CTAs in x).  No CTA leaves the kernel between
+  //      its start and here except through the window check above, which fails in all CTAs or in none; so every CTA
+  //      reaches both barriers.  After the first, CTA `slice` adds, for its share of the block's rows, the sums of
+  //      all slices in slice order straight out of the other CTAs' shared memory, applies the codebook and stores;
+  //      the second keeps every CTA's shared memory alive until all have read it.
+  __syncthreads();
+  cluster_sync_all();
+  {
+    const int share = (rows_blk + slices - 1) / slices;
+    const int r_begin = slice * share, r_end = min(rows_blk, r_begin + share);
+    float sx = 0.f;
+    for (int s2 = 0; s2 < slices; ++s2) sx += ld_cluster_f32(wb + G::kSxWord, (uint32_t)s2);
+    for (int row_local = r_begin + (int)threadIdx.x; row_local < r_end; row_local += (int)blockDim.x) {
+      const int64_t n = (int64_t)t0 * 16 + row_local;
+      if (n >= N) break;
+      uint32_t c[2];
+      load_row_codebook<BITS>(cb, n, c);
+      float a[CL];
+#pragma unroll
+      for (int q = 0; q < CL; ++q) a[q] = 0.f;
+      for (int s2 = 0; s2 < slices; ++s2) {
+#pragma unroll
+        for (int q = 0; q < CL; ++q)
+          a[q] += ld_cluster_f32(wb + G::kPartBase + 4u * (uint32_t)(q * rows_blk + row_local), (uint32_t)s2);
+      }
+      const int sm = smallest_centroid<BITS>(c);
+      auto cent = [&](int i) { return bf16_bits_to_float((c[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu); };
+      const float cs = cent(sm);
+      float out = cs * sx;
+#pragma unroll
+      for (int q = 0; q < CL; ++q) out = fmaf(cent(sm ^ (q + 1)) - cs, a[q], out);
+      y[n] = (uint16_t)float_to_bf16_bits(out);
+    }
+  }
+  cluster_sync_all();
 }
 
 // Second kernel (more than one slice): adds the slices of every row in a fixed order, applies the codebook and stores
@@ -428,33 +501,98 @@ namespace {
 
 struct LutPlan {
   int nl, slices, row_blocks, warps;
+  int cluster;   // 1: the slices of a row block form a thread-block cluster and are added through its shared memory
 };
 
 constexpr int lut_max_warps(int nl) { return nl <= 2 ? 32 : nl == 3 ? 24 : 20; }
 
+// How many clusters of `csize` CTAs of linear_lut_kernel<BITS, NL> can be resident at once (0: none, or the query
+// failed).
+template <int BITS, int NL>
+int lut_cluster_capacity_one(int csize) {
+  using G = LutGeo<BITS, NL>;
+  constexpr int smem = (int)G::kHighEnd - 1024;
+  if (cudaFuncSetAttribute(linear_lut_kernel<BITS, NL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+    return 0;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)csize;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(csize * 64));
+  cfg.blockDim = dim3((unsigned)(G::kWarps * 32));
+  cfg.dynamicSmemBytes = smem;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, linear_lut_kernel<BITS, NL>, &cfg) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return 0;
+  }
+  return n;
+}
+
+int lut_cluster_capacity(int bits, int nl, int csize) {
+  static int cache[64][3][5][4];   // [device][bits][nl][log2 csize]; 0 = not asked yet, -1 = none
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  const int lg = csize == 2 ? 1 : csize == 4 ? 2 : csize == 8 ? 3 : 0;
+  if (lg == 0 || nl < 1 || nl > 4 || (bits != 1 && bits != 2) || (bits == 2 && nl > 3)) return 0;
+  std::lock_guard<std::mutex> lock(mu);
+  int& c = cache[dev][bits][nl][lg];
+  if (c == 0) {
+    int n = 0;
+    if (bits == 1) n = nl == 1 ? lut_cluster_capacity_one<1, 1>(csize) : nl == 2 ? lut_cluster_capacity_one<1, 2>(csize)
+                     : nl == 3 ? lut_cluster_capacity_one<1, 3>(csize) : lut_cluster_capacity_one<1, 4>(csize);
+    else n = nl == 1 ? lut_cluster_capacity_one<2, 1>(csize) : nl == 2 ? lut_cluster_capacity_one<2, 2>(csize)
+                     : lut_cluster_capacity_one<2, 3>(csize);
+    c = n > 0 ? n : -1;
+  }
+  return c > 0 ? c : 0;
+}
+
+// Floats of partial sums a CTA can keep for the reduction over its cluster.
+int lut_part_floats(int bits, int nl) {
+  if (bits == 1) return nl == 1 ? LutGeo<1, 1>::kPartFloats : nl == 2 ? LutGeo<1, 2>::kPartFloats
+                        : nl == 3 ? LutGeo<1, 3>::kPartFloats : LutGeo<1, 4>::kPartFloats;
+  return nl == 1 ? LutGeo<2, 1>::kPartFloats : nl == 2 ? LutGeo<2, 2>::kPartFloats : LutGeo<2, 3>::kPartFloats;
+}
+
 // Chunks per slice: the choice that minimises the shared-memory work of the busiest CTA (table build: 256 cycles per
 // chunk; lookups: 16 cycles per tile, chunk and class) with all CTAs resident at once; then as many warps as give
-// every warp the same number of tiles (at least 16: the table build needs them).
+// every warp the same number of tiles (at least 16: the table build needs them).  Adding the slices costs a second
+// kernel (about 5000 cycles with its two kernel-to-kernel transitions) unless the 2, 4 or 8 slices of a row block can
+// run as one cluster (about 1000 cycles for its two barriers and the loads from the other CTAs' shared memory).
 LutPlan plan_lut(int64_t N, int64_t K, int bits, int sm_count) {
   const int64_t chunks = table_chunks(K), tiles = table_tiles(N);
   const int classes = bits == 1 ? 1 : 3;
-  LutPlan best = {1, (int)chunks, 1, 16};
+  LutPlan best = {1, (int)chunks, 1, 16, 0};
   double best_cost = 1e30;
-  for (int nl = 1; nl <= (bits == 1 ? 4 : 3); ++nl) {
-    const int64_t slices = (chunks + nl - 1) / nl;
-    int64_t rb = sm_count / slices;
-    if (rb < 1) rb = 1;
-    if (rb > tiles) rb = tiles;
+  auto consider = [&](int nl, int64_t slices, int64_t rb, int cluster) {
     const int64_t tiles_cta = (tiles + rb - 1) / rb;
     const int64_t waves = (slices * rb + sm_count - 1) / sm_count;
     const int64_t tasks_warp = (tiles_cta + lut_max_warps(nl) - 1) / lut_max_warps(nl);
     int64_t warps = (tiles_cta + tasks_warp - 1) / tasks_warp;
     if (warps < 16) warps = 16;
     const double cost = (double)waves * (256.0 * nl + (16.0 * classes + 4.0) * nl * (double)(tasks_warp * warps) + 600.0) +
-                        8.0 * slices;
+                        8.0 * slices + (slices == 1 ? 0.0 : cluster ? 1000.0 : 5000.0);
     if (cost < best_cost) {
       best_cost = cost;
-      best = {nl, (int)slices, (int)rb, (int)warps};
+      best = {nl, (int)slices, (int)rb, (int)warps, cluster};
+    }
+  };
+  for (int nl = 1; nl <= (bits == 1 ? 4 : 3); ++nl) {
+    const int64_t slices = (chunks + nl - 1) / nl;
+    int64_t rb = sm_count / slices;
+    if (rb < 1) rb = 1;
+    if (rb > tiles) rb = tiles;
+    consider(nl, slices, rb, 0);
+    if (slices == 2 || slices == 4 || slices == 8) {
+      int64_t rbc = lut_cluster_capacity(bits, nl, (int)slices);
+      if (rbc > tiles) rbc = tiles;
+      if (rbc >= 1 && ((tiles + rbc - 1) / rbc) * 16 * classes <= lut_part_floats(bits, nl)) consider(nl, slices, rbc, 1);
     }
   }
   return best;
@@ -473,19 +611,23 @@ cudaError_t launch_lut_one(const uint32_t* packed, const uint16_t* cb, const uin
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;   // CTAs slice 0 .. slices-1 of a row block are consecutive in x
+  attr[1].val.clusterDim.x = (unsigned)p.slices;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(p.slices * p.row_blocks));
   cfg.blockDim = dim3((unsigned)(p.warps * 32));
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = p.cluster ? 2 : 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, linear_lut_kernel<BITS, NL>, reinterpret_cast<const unsigned char*>(packed),
-                                     cb, x, y, scratch, N, K, p.slices, p.row_blocks, err);
-  if (e != cudaSuccess || p.slices == 1) return e;
+                                     cb, x, y, scratch, N, K, p.slices, p.row_blocks, err, p.cluster);
+  if (e != cudaSuccess || p.slices == 1 || p.cluster) return e;
   cudaLaunchConfig_t fin = {};
   fin.gridDim = dim3((unsigned)((N + 31) / 32));
   fin.blockDim = dim3(kFinWarps * 32);
@@ -521,18 +663,21 @@ bool linear_lut_supports(int64_t N, int64_t K, int bits, int64_t M) {
 }
 
 // Where the table kernel is the faster one.  It costs one pass per batch row (the tensor-core kernels cost about the
-// same for 1 to 8 rows) and a fixed few microseconds for the table build and the second kernel, so it pays at batch 1
-// on large 1-bit layers (measured on B200: 8192 x 28672: 14.8 against 23.9 us; 8192 x 8192: 7.8 against 7.7 us;
-// b = 2, 8192 x 8192: 11.7 against 11.4 us).
+// same for 1 to 8 rows) and a fixed few microseconds (its CTAs take a whole SM each, so consecutive calls do not
+// overlap; the table build; the second kernel or the cluster reduction), so it pays at batch 1 on large 1-bit
+// layers.  Measured on B200, table against tensor-core kernel, b = 1, us per call: 8192 x 28672: 14.8 / 27.9;
+// 6144 x 20480: 10.0 / 15.9; 20480 x 6144: 10.6 / 14.6; 8192 x 8192: 8.0 / 9.1; at 50 to 59 M weights about equal
+// (4096 x 14336: 7.8 / 8.2; 14336 x 4096: 8.5 / 8.3; 8192 x 6144: 7.2 / 7.1; 16384 x 3072: 6.8 / 7.9); below, the
+// tensor-core kernel (6144 x 6144: 6.8 / 5.7; 4096 x 4096: 5.5 / 3.2).  b = 2 never: 8192 x 8192: 12.0 / 10.4.
 bool linear_lut_preferred(int64_t N, int64_t K, int bits, int64_t M) {
-  return linear_lut_supports(N, K, bits, M) && bits == 1 && M == 1 && N * K >= (int64_t(1) << 27);
+  return linear_lut_supports(N, K, bits, M) && bits == 1 && M == 1 && N * K >= (int64_t(1) << 26);
 }
 
 size_t linear_lut_scratch_bytes(int64_t N, int64_t K, int bits) {
   const DeviceInfo* di = device_info();
   if (!di) return 0;
   const LutPlan p = plan_lut(N, K, bits, di->sm_count);
-  if (p.slices == 1) return 0;   // every CTA sees the whole of K: nothing to exchange
+  if (p.slices == 1 || p.cluster) return 0;   // the whole of K in one CTA, or the slices added inside a cluster
   return lut_scratch_floats(p.slices, bits == 1 ? 1 : 3, table_tiles(N) * 16) * sizeof(float);
 }
 
