@@ -101,3 +101,25 @@ def test_every_b1_b2_variant_was_reached():
                     names.add(kmq.kmq_linear_variant(64, K, bits, M, layout))
     for want in ("tiled_", "multi_", "staged_", "table_lookup_"):
         assert any(n.startswith(want) for n in names), f"no case reaches a {want}* kernel: {sorted(names)}"
+
+
+@pytest.mark.parametrize("M", (1, 2))
+@pytest.mark.parametrize("N,K", ((16, 512), (50, 1024), (700, 2048), (4096 + 7, 4096), (130, 6144 + 256), (9216, 3072)))
+@pytest.mark.parametrize("bits", (1, 2))
+def test_table_kernel_with_the_slices_of_a_row_block_as_one_cluster(bits, N, K, M):
+    """Shapes whose K range splits into 2, 4 or 8 slices: the table kernel then adds the slices inside a thread-block
+    cluster (one launch, no scratch).  Ragged row counts, more row blocks than one, skewed codebooks on the first
+    rows; the output must not depend on which of the two forms ran."""
+    if kmq.kmq_workspace_bytes(N, K, bits, M, L) != 0 or kmq.kmq_linear_num_launches(N, K, bits, M, L) != M:
+        pytest.skip("the planner adds the slices with a second kernel for this shape on this device")
+    rng = np.random.default_rng(bits * 100 + N + K + M)
+    Q = 1 << bits
+    idx = rng.integers(0, Q, size=(N, K), dtype=np.uint8)
+    cbv = np.sort(rng.standard_normal((N, Q)) * 0.02, axis=1)
+    sk = skewed_codebooks(bits)
+    for i, c in enumerate(sk[:min(N, len(sk))]):
+        cbv[i] = c
+        idx[i] = i % Q
+    cb = bf16(cbv)
+    x = bf16(rng.standard_normal((M, K)) * 2.0 ** rng.uniform(-8, 3, size=(M, K)))
+    assert check(idx, cb, x, bits, L).startswith("table_lookup")
