@@ -22,11 +22,43 @@ __device__ __forceinline__ double value_of(uint32_t k) {
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// Fit.  One CTA per row: the row is sorted once in shared memory (bitonic network on the keys); a fixed two-level
-// float64 prefix sum over chunks of 32 sorted values then gives the sum of any run of sorted values, so that an
-// iteration is one binary search and one partial chunk per cluster boundary.  The clusters of 1-D Lloyd are runs of
-// the sorted row: cluster i holds the values in (mid_{i-1}, mid_i], mid_i = (c_i + c_{i+1}) / 2 in float64.
+// Fit.  One CTA per row: the row is sorted once (bitonic network on the keys); a fixed two-level float64 prefix sum
+// over chunks of 32 sorted values then gives the sum of any run of sorted values, so that an iteration is one binary
+// search and one partial chunk per cluster boundary.  The clusters of 1-D Lloyd are runs of the sorted row: cluster i
+// holds the values in (mid_{i-1}, mid_i], mid_i = (c_i + c_{i+1}) / 2 in float64.
+//
+// The sort keeps 32 keys per thread in registers: key number i of the (padded) row sits in register i % 32 of lane
+// (i / 32) % 32 of warp i / 1024.  A compare-exchange at distance below 32 is then a register pair of one thread, at
+// distance 32 .. 512 a warp shuffle, and only at distance 1024 and above an exchange through shared memory.  The
+// direction of a merge phase is the same for all keys of a thread once the runs are 32 or longer; a thread whose
+// runs go downwards complements its keys for the phase and merges upwards like everybody else.
+// Shared memory holds key i at word i + i / 32: a thread's 32 keys and the same register of 32 lanes both fall on 32
+// different banks.
 // ---------------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ int phys(int i) { return i + (i >> 5); }
+
+// compare-exchange of registers at distance 2^B; ascending where bit M of the register number is clear (M > 4: always)
+template <int B, int M>
+__device__ __forceinline__ void local_stage(uint32_t (&k)[32]) {
+#pragma unroll
+  for (int r = 0; r < 32; ++r) {
+    if ((r >> B) & 1) continue;
+    const uint32_t a = k[r], b = k[r | (1 << B)];
+    const bool up = M > 4 || ((r >> M) & 1) == 0;
+    k[r] = up ? min(a, b) : max(a, b);
+    k[r | (1 << B)] = up ? max(a, b) : min(a, b);
+  }
+}
+
+// the five stages at distances 16 .. 1, all ascending
+__device__ __forceinline__ void local_merge(uint32_t (&k)[32]) {
+  local_stage<4, 5>(k);
+  local_stage<3, 5>(k);
+  local_stage<2, 5>(k);
+  local_stage<1, 5>(k);
+  local_stage<0, 5>(k);
+}
+
 __global__ void __launch_bounds__(1024) lloyd_rows_kernel(const float* __restrict__ W, int64_t N, int64_t K, int Q,
                                                           int iters, int P, uint16_t* __restrict__ codebooks,
                                                           double* __restrict__ centroids) {
@@ -36,35 +68,69 @@ __global__ void __launch_bounds__(1024) lloyd_rows_kernel(const float* __restric
   double* pre = c + kMaxCentroids;                               // [257] prefix sum at each cluster boundary
   double* wtot = pre + kMaxCentroids + 1;                        // [32] warp totals of the scan
   int* edge = reinterpret_cast<int*>(wtot + 32);                 // [258] cluster boundaries (sorted positions)
-  uint32_t* keys = reinterpret_cast<uint32_t*>(edge + 258);      // [P]
+  uint32_t* keys = reinterpret_cast<uint32_t*>(edge + 258);      // [P + P / 32], key i at phys(i)
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
   const int Kc = (int)K, chunks = (Kc + 31) >> 5;
+  int logP = 10;
+  while ((1 << logP) < P) ++logP;                                // P = 32 * nthr = 2^logP >= 1024
 
   for (int64_t row = blockIdx.x; row < N; row += gridDim.x) {
     const float* w = W + row * K;
-    for (int i = tid; i < P; i += nthr) keys[i] = i < Kc ? key_of(w[i]) : 0xFFFFFFFFu;
+    for (int i = tid; i < P; i += nthr) keys[phys(i)] = i < Kc ? key_of(w[i]) : 0xFFFFFFFFu;   // coalesced reads
     __syncthreads();
-    for (int k = 2; k <= P; k <<= 1) {
-      for (int j = k >> 1; j > 0; j >>= 1) {
-        for (int t = tid; t < (P >> 1); t += nthr) {
-          const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1)), p = i | j;
-          const uint32_t a = keys[i], b = keys[p];
-          const uint32_t lo = min(a, b), hi = max(a, b);
-          const bool up = (i & k) == 0;
-          keys[i] = up ? lo : hi;
-          keys[p] = up ? hi : lo;
-        }
+    uint32_t k[32];
+#pragma unroll
+    for (int r = 0; r < 32; ++r) k[r] = keys[phys((tid << 5) + r)];
+    // runs of 2, 4, 8, 16 inside the thread, directions by the register number
+    local_stage<0, 1>(k);
+    local_stage<1, 2>(k);
+    local_stage<0, 2>(k);
+    local_stage<2, 3>(k);
+    local_stage<1, 3>(k);
+    local_stage<0, 3>(k);
+    local_stage<3, 4>(k);
+    local_stage<2, 4>(k);
+    local_stage<1, 4>(k);
+    local_stage<0, 4>(k);
+    // phases m = 5 .. logP: runs of 2^m, direction by bit m of the key number (clear in the last phase)
+    for (int m = 5; m <= logP; ++m) {
+      const uint32_t flip = (((tid << 5) >> m) & 1) ? 0xFFFFFFFFu : 0u;
+#pragma unroll
+      for (int r = 0; r < 32; ++r) k[r] ^= flip;
+      for (int b = m - 1; b >= 10; --b) {          // partner in another warp: through shared memory
+        __syncthreads();                            // the previous readers of `keys` are done
+#pragma unroll
+        for (int r = 0; r < 32; ++r) keys[phys((tid << 5) + r)] = k[r];
         __syncthreads();
+        const int partner = (tid ^ (1 << (b - 5))) << 5;
+        const bool lower = ((tid >> (b - 5)) & 1) == 0;
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+          const uint32_t o = keys[phys(partner + r)];
+          k[r] = lower ? min(k[r], o) : max(k[r], o);
+        }
       }
+      for (int b = (m - 1 < 9 ? m - 1 : 9); b >= 5; --b) {   // partner in another lane: shuffle
+        const int d = 1 << (b - 5);
+        const bool lower = (lane & d) == 0;
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+          const uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, k[r], d);
+          k[r] = lower ? min(k[r], o) : max(k[r], o);
+        }
+      }
+      local_merge(k);
+#pragma unroll
+      for (int r = 0; r < 32; ++r) k[r] ^= flip;
     }
-    // chunk sums (thread t owns sorted positions [32t, 32t + 32); rotated start: no bank conflicts) and their scan
+    // the sorted row goes back to shared memory; chunk t = the 32 keys of thread t: its float64 sum, then the scan
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 32; ++r) keys[phys((tid << 5) + r)] = k[r];
     double v = 0.0;
-    if (tid < chunks) {
-      for (int jj = 0; jj < 32; ++jj) {
-        const int pos = (tid << 5) + ((jj + tid) & 31);
-        if (pos < Kc) v = __dadd_rn(v, value_of(keys[pos]));
-      }
-    }
+#pragma unroll
+    for (int r = 0; r < 32; ++r)
+      if ((tid << 5) + r < Kc) v = __dadd_rn(v, value_of(k[r]));
     double incl = v;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -92,43 +158,60 @@ __global__ void __launch_bounds__(1024) lloyd_rows_kernel(const float* __restric
       if (tid == chunks - 1) cpre[chunks] = __dadd_rn(excl, v);
     }
     // start: linearly interpolated order statistics at (i + 1/2) / Q
-    if (tid < Q) {
-      const double pos = __dmul_rn(__ddiv_rn((double)tid + 0.5, (double)Q), (double)(Kc - 1));
+    for (int j = tid; j < Q; j += nthr) {
+      const double pos = __dmul_rn(__ddiv_rn((double)j + 0.5, (double)Q), (double)(Kc - 1));
       const int lo = (int)floor(pos), hi = min(lo + 1, Kc - 1);
       const double t = __dadd_rn(pos, -(double)lo);
-      c[tid] = __dadd_rn(__dmul_rn(value_of(keys[lo]), __dadd_rn(1.0, -t)), __dmul_rn(value_of(keys[hi]), t));
+      c[j] = __dadd_rn(__dmul_rn(value_of(keys[phys(lo)]), __dadd_rn(1.0, -t)), __dmul_rn(value_of(keys[phys(hi)]), t));
     }
     __syncthreads();
     for (int it = 0; it < iters; ++it) {
-      for (int i = warp; i < Q - 1; i += nwarps) {
-        const double mid = __dmul_rn(0.5, __dadd_rn(c[i], c[i + 1]));
-        int lo = 0, hi = Kc;                      // first sorted position whose value is above mid
-        while (lo < hi) {
-          const int m = (lo + hi) >> 1;
-          if (value_of(keys[m]) <= mid) lo = m + 1;
-          else hi = m;
-        }
-        const int base = lo & ~31;
-        double part = (base + lane < lo) ? value_of(keys[base + lane]) : 0.0;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) part = __dadd_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, d));
-        if (lane == 0) {
+      if (Q - 1 > nwarps) {
+        // more cluster boundaries than warps: a thread per boundary (the partial chunk added in index order)
+        for (int i = tid; i < Q - 1; i += nthr) {
+          const double mid = __dmul_rn(0.5, __dadd_rn(c[i], c[i + 1]));
+          int lo = 0, hi = Kc;                      // first sorted position whose value is above mid
+          while (lo < hi) {
+            const int m = (lo + hi) >> 1;
+            if (value_of(keys[phys(m)]) <= mid) lo = m + 1;
+            else hi = m;
+          }
+          double part = 0.0;
+          for (int j = lo & ~31; j < lo; ++j) part = __dadd_rn(part, value_of(keys[phys(j)]));
           edge[i + 1] = lo;
           pre[i + 1] = __dadd_rn(cpre[lo >> 5], part);
         }
+      } else {
+        for (int i = warp; i < Q - 1; i += nwarps) {   // a warp per boundary
+          const double mid = __dmul_rn(0.5, __dadd_rn(c[i], c[i + 1]));
+          int lo = 0, hi = Kc;                      // first sorted position whose value is above mid
+          while (lo < hi) {
+            const int m = (lo + hi) >> 1;
+            if (value_of(keys[phys(m)]) <= mid) lo = m + 1;
+            else hi = m;
+          }
+          const int base = lo & ~31;
+          double part = (base + lane < lo) ? value_of(keys[phys(base + lane)]) : 0.0;
+#pragma unroll
+          for (int d = 16; d > 0; d >>= 1) part = __dadd_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, d));
+          if (lane == 0) {
+            edge[i + 1] = lo;
+            pre[i + 1] = __dadd_rn(cpre[lo >> 5], part);
+          }
+        }
       }
       __syncthreads();
-      if (tid < Q) {
-        const int e0 = tid == 0 ? 0 : edge[tid], e1 = tid == Q - 1 ? Kc : edge[tid + 1];
-        const double p0 = tid == 0 ? 0.0 : pre[tid], p1 = tid == Q - 1 ? cpre[chunks] : pre[tid + 1];
-        if (e1 > e0) c[tid] = __ddiv_rn(__dadd_rn(p1, -p0), (double)(e1 - e0));
+      for (int j = tid; j < Q; j += nthr) {
+        const int e0 = j == 0 ? 0 : edge[j], e1 = j == Q - 1 ? Kc : edge[j + 1];
+        const double p0 = j == 0 ? 0.0 : pre[j], p1 = j == Q - 1 ? cpre[chunks] : pre[j + 1];
+        if (e1 > e0) c[j] = __ddiv_rn(__dadd_rn(p1, -p0), (double)(e1 - e0));
       }
       __syncthreads();
     }
-    if (tid < Q) {
-      if (centroids) centroids[row * Q + tid] = c[tid];
-      const uint32_t stored = float_to_bf16_bits(__double2float_rn(c[tid]));
-      codebooks[row * Q + tid] = (uint16_t)((stored & 0x7FFFu) ? stored : 0u);   // a zero centroid is stored as +0
+    for (int j = tid; j < Q; j += nthr) {
+      if (centroids) centroids[row * Q + j] = c[j];
+      const uint32_t stored = float_to_bf16_bits(__double2float_rn(c[j]));
+      codebooks[row * Q + j] = (uint16_t)((stored & 0x7FFFu) ? stored : 0u);   // a zero centroid is stored as +0
     }
     __syncthreads();
   }
@@ -401,7 +484,9 @@ cudaError_t launch_assign_bits(const float* W, const uint16_t* cb, int64_t N, in
 
 }  // namespace
 
-size_t fit_smem_bytes(int P) { return (size_t)(1025 + kMaxCentroids + kMaxCentroids + 1 + 32) * 8 + 258 * 4 + (size_t)P * 4; }
+size_t fit_smem_bytes(int P) {
+  return (size_t)(1025 + kMaxCentroids + kMaxCentroids + 1 + 32) * 8 + 258 * 4 + (size_t)(P + P / 32) * 4;
+}
 
 bool fit_supports(int64_t K, int bits) { return K >= (int64_t(1) << bits) && K >= 2 && K <= kMaxFitLen; }
 
@@ -409,9 +494,9 @@ cudaError_t launch_kmeans_rows(const float* W, int64_t N, int64_t K, int bits, i
                                double* centroids, cudaStream_t s) {
   const DeviceInfo* di = device_info();
   if (!di) return cudaErrorInvalidDevice;
-  int P = 64;
+  int P = 1024;                      // keys sorted, padded: a power of two, 32 per thread
   while (P < K) P <<= 1;
-  const int threads = P / 2 < 64 ? 64 : (P / 2 > 1024 ? 1024 : P / 2);
+  const int threads = P / 32;
   const size_t smem = fit_smem_bytes(P);
   if (cudaError_t e = cudaFuncSetAttribute(lloyd_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)fit_smem_bytes(kMaxFitLen)))

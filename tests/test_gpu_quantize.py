@@ -84,7 +84,7 @@ def test_kmeans_rows_matches_the_oracle(bits, K, dist):
     check_fit(draw_rows(dist, 20, K, 7 * bits + K), bits)
 
 
-@pytest.mark.parametrize("bits,K,N", ((1, 28672, 3), (4, 28672, 3), (8, 32768, 1), (8, 5000, 2), (2, 2, 3), (1, 3, 2)))
+@pytest.mark.parametrize("bits,K,N", ((1, 28672, 3), (4, 28672, 3), (8, 32768, 1), (8, 5000, 2), (8, 256, 2), (8, 300, 1), (4, 1024, 2), (4, 1025, 2), (2, 2, 3), (1, 3, 2)))
 def test_kmeans_rows_long_short_and_8_bit(bits, K, N):
     if K < (1 << bits):
         pytest.skip("fewer values than centroids")
