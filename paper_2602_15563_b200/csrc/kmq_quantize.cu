@@ -63,12 +63,13 @@ __global__ void __launch_bounds__(1024) lloyd_rows_kernel(const float* __restric
                                                           int iters, int P, uint16_t* __restrict__ codebooks,
                                                           double* __restrict__ centroids) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* cpre = reinterpret_cast<double*>(smem_raw);            // [1025] exclusive prefix of the chunk sums
-  double* c = cpre + 1025;                                       // [256] centroids
-  double* pre = c + kMaxCentroids;                               // [257] prefix sum at each cluster boundary
-  double* wtot = pre + kMaxCentroids + 1;                        // [32] warp totals of the scan
-  int* edge = reinterpret_cast<int*>(wtot + 32);                 // [258] cluster boundaries (sorted positions)
-  uint32_t* keys = reinterpret_cast<uint32_t*>(edge + 258);      // [P + P / 32], key i at phys(i)
+  // sized by the launch: P / 32 chunks, Q centroids (fit_smem_bytes)
+  double* cpre = reinterpret_cast<double*>(smem_raw);            // [P / 32 + 1] exclusive prefix of the chunk sums
+  double* c = cpre + (P >> 5) + 1;                               // [Q] centroids
+  double* pre = c + Q;                                           // [Q + 1] prefix sum at each cluster boundary
+  double* wtot = pre + Q + 1;                                    // [32] warp totals of the scan
+  int* edge = reinterpret_cast<int*>(wtot + 32);                 // [Q + 2] cluster boundaries (sorted positions)
+  uint32_t* keys = reinterpret_cast<uint32_t*>(edge + Q + 2);    // [P + P / 32], key i at phys(i)
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
   const int Kc = (int)K, chunks = (Kc + 31) >> 5;
   int logP = 10;
@@ -484,8 +485,8 @@ cudaError_t launch_assign_bits(const float* W, const uint16_t* cb, int64_t N, in
 
 }  // namespace
 
-size_t fit_smem_bytes(int P) {
-  return (size_t)(1025 + kMaxCentroids + kMaxCentroids + 1 + 32) * 8 + 258 * 4 + (size_t)(P + P / 32) * 4;
+size_t fit_smem_bytes(int P, int Q) {
+  return (size_t)((P >> 5) + 1 + Q + Q + 1 + 32) * 8 + (size_t)(Q + 2) * 4 + (size_t)(P + P / 32) * 4;
 }
 
 bool fit_supports(int64_t K, int bits) { return K >= (int64_t(1) << bits) && K >= 2 && K <= kMaxFitLen; }
@@ -497,9 +498,9 @@ cudaError_t launch_kmeans_rows(const float* W, int64_t N, int64_t K, int bits, i
   int P = 1024;                      // keys sorted, padded: a power of two, 32 per thread
   while (P < K) P <<= 1;
   const int threads = P / 32;
-  const size_t smem = fit_smem_bytes(P);
+  const size_t smem = fit_smem_bytes(P, 1 << bits);
   if (cudaError_t e = cudaFuncSetAttribute(lloyd_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)fit_smem_bytes(kMaxFitLen)))
+                                           (int)fit_smem_bytes(kMaxFitLen, kMaxCentroids)))
     return e;
   int per_sm = 1;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, lloyd_rows_kernel, threads, smem) != cudaSuccess || per_sm < 1)
