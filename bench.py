@@ -301,11 +301,13 @@ PAPER_TOKENS_PER_S = {"decode_4b": {16: 88.8, 4.25: 190.1, 1.25: 245.6}, "decode
                       "decode_31b": {4.25: 35.4, 1.25: 60.7}}
 
 
-def decode_layer_shapes(model):
+def decode_layer_shapes(model, fused_gate_up=False):
     d, L, heads, kv = DECODE_MODELS[model]
     hidden = -(-int(1.3 * 8 * d / 3) // 1024) * 1024
     qkv = (heads + 2 * kv) * 128
     # (name, N out, K in, input: index of the call of the same layer whose output it reads, or -1 = the layer input)
+    if fused_gate_up:    # the gate and up matrices stacked along N (they read the same input): one call
+        return L, [("qkv", qkv, d, -1), ("o", d, d, 0), ("gate_up", 2 * hidden, d, 1), ("down", d, hidden, 2)]
     return L, [("qkv", qkv, d, -1), ("o", d, d, 0), ("gate", hidden, d, 1), ("up", hidden, d, 1), ("down", d, hidden, 2)]
 
 
@@ -333,7 +335,8 @@ def run_decode(args):
     sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
     sampler.start()
     stream = torch.cuda.Stream()
-    for bits in (1, 4):
+    for fused, bits in ((False, 1), (False, 4), (True, 1), (True, 4)):
+        L, shapes = decode_layer_shapes(args.workload, fused)
         g = torch.Generator(device=dev).manual_seed(bits)
         calls, step_bytes, ws_bytes = [], 0, 16
         x0 = (torch.randn(d, device=dev, generator=g)).to(torch.bfloat16).view(torch.int16)
@@ -398,7 +401,7 @@ def run_decode(args):
             sampler.active = False
         ms = e0.elapsed_time(e1) / steps
         variants = sorted({f"{c['name']}:{c['variant']}" for c in calls[:len(shapes)]})
-        results.append({"bits": bits, "ms_per_token": round(ms, 4), "tokens_per_s_equivalent": round(1e3 / ms, 1),
+        results.append({"bits": bits, "gate_up": "one call" if fused else "two calls", "ms_per_token": round(ms, 4), "tokens_per_s_equivalent": round(1e3 / ms, 1),
                         "gbs": round(step_bytes / (ms * 1e-3) / 1e9, 1),
                         "frac_of_measured_hbm": round(step_bytes / (ms * 1e-3) / 1e9 / peak_gbs, 4),
                         "calls_per_token": len(calls), "launches_per_token": sum(c["launches"] for c in calls),
@@ -407,6 +410,7 @@ def run_decode(args):
         del calls, outs, ws, graph
         torch.cuda.empty_cache()
     sampler.stop_flag = True
+    L, shapes = decode_layer_shapes(args.workload)
     best = max(results, key=lambda r: r["gbs"])
     line = {
         "metric": "kmq_linear effective HBM bandwidth (algorithmic bytes / time), batch-1 k-means LUT GEMV",
@@ -415,7 +419,8 @@ def run_decode(args):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{args.workload}: every backbone linear of one decoding step at batch 1, "
                                f"L = {L} layers x {[(n, N, K) for (n, N, K, _s) in shapes]}, one CUDA graph per token, "
-                               "distinct weights per matrix (far larger than L2), random indices",
+                               "distinct weights per matrix (far larger than L2), random indices; timed a second time with "
+                               "the gate and up matrices stacked into one call (per_bits: gate_up)",
                    "multi_gpu": "replicas only"},
         "per_bits": results,
         "roofline": {"bound": "hbm", "kernel": "all kmq_linear calls of a token", "achieved": best["gbs"],
