@@ -64,7 +64,8 @@ __device__ __forceinline__ int piece_offset(int w) {
 template <int BITS, int MMAX>
 __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed, const uint16_t* __restrict__ cb,
                                              const uint16_t* __restrict__ x, int64_t N, int64_t K, int M,
-                                             int64_t tile_id, int sa, int sb, bool wait_for_x, float& v) {
+                                             int64_t tile_id, int sa, int sb, bool wait_for_x, bool early_trigger,
+                                             float& v) {
   using G = TGeo<BITS>;
   using SM = TSmem<BITS, MMAX>;
   constexpr int Q = G::kMmaPerWord;
@@ -167,6 +168,9 @@ __device__ __forceinline__ void tile_segment(const uint32_t* __restrict__ packed
         asm volatile("prefetch.global.L2 [%0];" ::"l"(x + o));
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Where it pays (see early_trigger()), the next kernel on the stream may become resident from here on: its CTAs
+    // read their packed words and build their tables in the SM slots this grid leaves free, while this one computes.
+    if (early_trigger) asm volatile("griddepcontrol.launch_dependents;");
   }
   if constexpr (kPrefetchX) {
 #pragma unroll
@@ -270,14 +274,14 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) linear_tiled_kernel(c
                                                                     const uint16_t* __restrict__ cb,
                                                                     const uint16_t* __restrict__ x,
                                                                     uint16_t* __restrict__ y, int64_t N, int64_t K,
-                                                                    int M) {
+                                                                    int M, int early) {
   const int steps = (int)((K / (4 * TGeo<BITS>::kWordK) + 3) >> 2);
   const int64_t row0 = (int64_t)blockIdx.x * kRows;
   float v;
-  tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, blockIdx.x, 0, steps, true, v);
-  // Programmatic dependent launch: from here on the next kernel on the stream may become resident; it reads nothing
-  // but constants of its layer until this kernel has completed (see tile_segment), so its first weights are under
-  // way while this one stores and drains.
+  tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, blockIdx.x, 0, steps, true, early != 0, v);
+  // Programmatic dependent launch: from here on at the latest the next kernel on the stream may become resident; it
+  // reads nothing but constants of its layer until this kernel has completed (see tile_segment), so its first
+  // weights are under way while this one stores and drains.
   asm volatile("griddepcontrol.launch_dependents;");
   store_output(v, y, N, M, row0);
 }
@@ -304,7 +308,7 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) linear_split_kernel(c
     const int64_t base = tile * steps;
     const int sa = (int)(u0 > base ? u0 - base : 0), sb = (int)(u1 - base < steps ? u1 - base : steps);
     float v;
-    tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, tile, sa, sb, false, v);
+    tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, tile, sa, sb, false, false, v);
     if (sa == 0 && sb == steps) {
       store_output(v, y, N, M, tile * kRows);
     } else if (threadIdx.x < kRows * 8) {
@@ -331,6 +335,24 @@ __global__ void __launch_bounds__(kRows * 8) linear_split_fixup_kernel(const flo
   store_output(v, y, N, M, row0);
 }
 
+// Whether the CTAs of linear_tiled_kernel release the next kernel on the stream right after their own wait instead of
+// just before their store.  The next call's CTAs then take the SM slots this grid leaves free and do their set-up
+// (packed words, b = 4 tables) under this grid's MMAs, at the price of competing with them.  Measured on B200 at
+// batch 1 over N = 2048 .. 16384, K = 2048 .. 11264 (us per call, late / early release):
+//   b = 2: faster nearly everywhere (4096 x 4096 3.64 / 3.25, 3072 x 3072 2.94 / 2.68, 8192 x 8192 10.4 / 9.9) except
+//          with between two and three CTAs per SM (5120 x 4096 4.68 / 4.99, 6144 x 4096 4.83 / 5.08);
+//   b = 4: faster (5120 x 4096 6.61 / 5.46, 3072 x 3072 4.03 / 3.46, 8192 x 8192 16.1 / 15.4) except when the grid
+//          nearly fills two CTA slots of every SM and tiles are long (4096 x 4096 4.92 / 5.13, 4096 x 8192 8.06 / 8.92);
+//   b = 1: no gain or a loss (4096 x 4096 3.14 / 3.90) except on long tiles away from that window (3072 x 8192
+//          5.15 / 4.83, 8192 x 8192 9.09 / 8.48).
+bool early_trigger(int bits, int64_t tiles, int64_t steps, int sm_count) {
+  const int64_t two = 2 * (int64_t)sm_count, three = 3 * (int64_t)sm_count;
+  const bool nearly_two = 5 * tiles > 4 * two && tiles <= two;   // more than 0.8 of two CTAs per SM, at most two
+  if (bits == 2) return !(tiles > two && tiles < three);
+  if (bits == 4) return !(nearly_two && steps >= 32);
+  return steps >= 16 && !(10 * tiles > 7 * two && tiles <= two);
+}
+
 template <int BITS, int MMAX>
 cudaError_t launch_one(const uint32_t* packed, const uint16_t* cb, const uint16_t* x, uint16_t* y, int64_t N,
                        int64_t K, int M, cudaStream_t s) {
@@ -354,7 +376,10 @@ cudaError_t launch_one(const uint32_t* packed, const uint16_t* cb, const uint16_
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, linear_tiled_kernel<BITS, MMAX>, packed, cb, x, y, N, K, M);
+  const DeviceInfo* di = device_info();
+  const int64_t steps = (K / (4 * TGeo<BITS>::kWordK) + 3) >> 2;
+  const int early = di && early_trigger(BITS, (N + kRows - 1) / kRows, steps, di->sm_count) ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, linear_tiled_kernel<BITS, MMAX>, packed, cb, x, y, N, K, M, early);
 }
 
 template <int BITS>
