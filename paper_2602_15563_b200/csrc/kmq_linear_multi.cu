@@ -119,8 +119,6 @@ __global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 
       qb[d] = ldg_stream_u4(tile + (int64_t)s * 64 + 32);
     }
   }
-  if (group < steps) stage(group, 0);
-
   // ---- per-row decode state ----
   Dec1 sg, sh;
   if constexpr (BITS == 1) {
@@ -142,6 +140,14 @@ __global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 
     }
     __syncthreads();
   }
+  // Programmatic dependent launch: up to here only the packed indices and the codebooks were read (constants of the
+  // layer); the activations may come from the previous kernel on the stream and are read only once it has completed.
+  // At b = 4, where the set-up of a CTA is long (its tables), the next kernel is released at once so that its CTAs
+  // set up under this grid's MMAs; otherwise just before the partial sums are exchanged (measured, 4096 x 4096 M = 16:
+  // b = 4 9.7 -> 8.3 us early, 8.7 late; b = 2 6.4 -> 6.3 / 6.5; 8192 x 8192 b = 2 M = 32 20.1 -> 20.1 / 19.5).
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if constexpr (BITS == 4) asm volatile("griddepcontrol.launch_dependents;");
+  if (group < steps) stage(group, 0);
   const unsigned char* const tab_g = tables + wt * kTableBytesPerTile;   // rows g; rows g + 8 are 2 KB further
   const uint32_t lane4 = lane * 4;
 
@@ -215,6 +221,7 @@ __global__ void __launch_bounds__(W * 32, (W == 8 && NT <= 2 && TPC == 2) ? 2 : 
   }
 
   // ---- K-groups 1.. hand their partial sums to K-group 0, which adds and stores ----
+  asm volatile("griddepcontrol.launch_dependents;");
   __syncthreads();   // every warp is done with the x buffers; `red` aliases them
   if (group > 0) {
 #pragma unroll
@@ -258,8 +265,17 @@ cudaError_t launch_nt(const uint32_t* packed, const uint16_t* cb, const uint16_t
   }
   const int64_t tiles = (N + kTileRows - 1) / kTileRows;
   const unsigned grid = (unsigned)((tiles + TPC - 1) / TPC);
-  linear_multi_kernel<BITS, NT, TPC, W><<<grid, W * 32, smem, s>>>(packed, cb, x, y, N, K, M);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(W * 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, linear_multi_kernel<BITS, NT, TPC, W>, packed, cb, x, y, N, K, M);
 }
 
 template <int BITS>

@@ -304,11 +304,13 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) linear_split_kernel(c
   const int64_t steps = (K / (4 * TGeo<BITS>::kWordK) + 3) >> 2;
   const int64_t units = ((N + kRows - 1) / kRows) * steps;
   const int64_t u0 = units * blockIdx.x / gridDim.x, u1 = units * (blockIdx.x + 1) / gridDim.x;
+  bool first = true;   // the first segment waits for the previous kernel on the stream before it reads x
   for (int64_t tile = u0 / steps; tile * steps < u1; ++tile) {
     const int64_t base = tile * steps;
     const int sa = (int)(u0 > base ? u0 - base : 0), sb = (int)(u1 - base < steps ? u1 - base : steps);
     float v;
-    tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, tile, sa, sb, false, false, v);
+    tile_segment<BITS, MMAX>(packed, cb, x, N, K, M, tile, sa, sb, first, false, v);
+    first = false;
     if (sa == 0 && sb == steps) {
       store_output(v, y, N, M, tile * kRows);
     } else if (threadIdx.x < kRows * 8) {
@@ -316,6 +318,7 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) linear_split_kernel(c
       slot[threadIdx.x] = v;
     }
   }
+  asm volatile("griddepcontrol.launch_dependents;");
 }
 
 // Block c adds the two halves of the tile that the cut between CTA c and CTA c + 1 falls into.
@@ -328,6 +331,8 @@ __global__ void __launch_bounds__(kRows * 8) linear_split_fixup_kernel(const flo
   const int64_t units = ((N + kRows - 1) / kRows) * steps;
   const int64_t cut = units * (blockIdx.x + 1) / ctas;
   if (cut % steps == 0) return;   // the cut is a tile boundary: nothing was left partial
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the slots are the previous kernel's output
+  asm volatile("griddepcontrol.launch_dependents;");
   const int64_t row0 = (cut / steps) * kRows;
   const float* end_of_c = scratch + ((int64_t)blockIdx.x * 2 + 1) * kSlotFloats;
   const float* start_of_next = scratch + ((int64_t)(blockIdx.x + 1) * 2) * kSlotFloats;
@@ -408,11 +413,25 @@ cudaError_t launch_split_one(const uint32_t* packed, const uint16_t* cb, const u
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  linear_split_kernel<BITS, MMAX><<<ctas, kThreads, smem, s>>>(packed, cb, x, y, N, K, M, scratch);
-  cudaError_t e = cudaGetLastError();
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)ctas);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, linear_split_kernel<BITS, MMAX>, packed, cb, x, y, N, K, M, scratch);
   if (e != cudaSuccess) return e;
-  linear_split_fixup_kernel<BITS><<<ctas - 1, kRows * 8, 0, s>>>(scratch, cb, y, N, K, M, ctas);
-  return cudaGetLastError();
+  cudaLaunchConfig_t fix = {};
+  fix.gridDim = dim3((unsigned)(ctas - 1));
+  fix.blockDim = dim3(kRows * 8);
+  fix.stream = s;
+  fix.attrs = attr;
+  fix.numAttrs = 1;
+  return cudaLaunchKernelEx(&fix, linear_split_fixup_kernel<BITS>, (const float*)scratch, cb, y, N, K, M, ctas);
 }
 
 template <int BITS>
