@@ -74,7 +74,7 @@ NCU_TRAFFIC_BYTES = {
     (4096, 4096, 4, 1, "tiled_pairtable_b4"): 8541184,
     (8192, 8192, 2, 1, "tiled_prmt_b2"): 16875008,          # profiles/kmq_linear_tiled_8192x8192_b2_ncu_full.md
     (8192, 28672, 1, 1, "table_lookup_b1"): 29493760 + 959488,            # main kernel + the kernel that adds the slices
-    (8192, 28672, 4, 1, "split_pairtable_b4"): 117777408 + 3555840 + 485888,   # main (read + scratch written) + fix-up
+    (8192, 28672, 4, 1, "split_pairtable_b4"): 117780992 + 4155392 + 486400,   # main (read + scratch written) + fix-up
 }
 
 
